@@ -305,3 +305,17 @@ def test_sgd_stationary_variance():
     S = O.State(w1, np.full(n, lam_v), np.zeros(n))
     S.run()
     assert S.theta[0].var() == pytest.approx(var / K, rel=0.05)
+
+
+def test_coordinate_subset_equals_the_same_columns_of_the_full_run():
+    """Coordinates never interact (diagonal loss, per-coordinate mean), so a run on a subset of columns, with the
+    noise addressed by the *global* coordinate index, reproduces those columns of the full run bit for bit."""
+    for opt in (W.OPT_SGDM, W.OPT_ADAMW):
+        w = W.tiny_workload(opt, K=3, P=203, T=30)
+        lam, ths = _inputs(w)
+        full = O.State(w, lam, ths)
+        full.run()
+        idx = np.array([0, 1, 5, 6, 7, 100, 201, 202], np.int64)
+        sub = O.State(w, lam[idx], ths[idx], idx=idx)
+        sub.run()
+        assert np.array_equal(sub.theta, full.theta[:, idx])
