@@ -1,0 +1,180 @@
+/*
+ * qsr.h -- C ABI of the Local-OPT / Quadratic-Synchronization-Rule hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library runs Algorithm 2 ("Local OPT") of "A Quadratic Synchronization Rule for Distributed Deep
+ * Learning" (arXiv 2310.14423) with the K workers laid out as the rows of [K, P] fp32 slabs in one GPU's
+ * memory: every worker takes local optimizer steps on its own stochastic gradient (Eq. 1), at the end of a
+ * round all workers replace their parameters by the mean over workers (the All-Reduce line of Algorithm 2,
+ * here a mean over the replica axis), and the length of each round follows Eq. 2.
+ *
+ * Conventions that hold for every call unless a comment says otherwise
+ *   - Pointers named params / state1 / state2 / grads / lambda / theta_star / sum / theta0_dev are DEVICE
+ *     pointers, 16-byte aligned; the caller owns them and keeps them alive until qsr_destroy.  The library
+ *     allocates no device memory and frees none.  Pointers with "host" in their name are HOST pointers.
+ *   - Slabs are row-major [K, row_stride] floats; worker k's coordinate i is slab[k * row_stride + i],
+ *     i < P <= row_stride, row_stride a multiple of 4.  Elements with i >= P are never read or written.
+ *   - Device work is enqueued on the CUDA stream given to qsr_init; no call waits for the device except
+ *     qsr_train_host.  The host-side schedule functions do no device work at all.
+ *   - Every function returns QSR_OK (0) or a negative qsr_status; none aborts, throws or exits.  A failed
+ *     call leaves the slabs untouched unless the failure is QSR_ECUDA from a launch.
+ *   - A context is used from one host thread at a time.
+ */
+#ifndef QSR_H_
+#define QSR_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct qsr_ctx qsr_ctx; /* opaque; host memory owned by the library */
+
+typedef enum {
+    QSR_OK = 0,
+    QSR_EINVAL = -1, /* NULL where a pointer is required, K < 1, P < 1, unknown enum value, non-finite number */
+    QSR_EALIGN = -2, /* a device pointer is not 16-byte aligned, or row_stride is not a multiple of 4 or < P */
+    QSR_ECUDA = -3,  /* the CUDA runtime reported an error (no device, launch failure, failed copy)          */
+    QSR_ERANGE = -4, /* t outside [0, T), T_warmup >= T, H_base < 1, K or t beyond 2^32, workspace too small */
+    QSR_ESTATE = -5  /* call out of order (e.g. qsr_sync_finish without qsr_sync_partial)                     */
+} qsr_status;
+
+enum { QSR_OPT_SGDM = 0, QSR_OPT_ADAMW = 1 };
+enum { QSR_SCHED_COSINE = 0, QSR_SCHED_STEP_POW2 = 1, QSR_SCHED_LINEAR = 2, QSR_SCHED_CONST = 3 };
+enum { QSR_RULE_QSR = 0, QSR_RULE_CONST_H = 1 };
+enum { QSR_STATE_KEEP = 0, QSR_STATE_AVERAGE = 1, QSR_STATE_RESET = 2 };
+
+/*
+ * One run.  Plain data; the library copies it.
+ *
+ * OPT (Eq. 1; hyper-parameters of App. C):
+ *   QSR_OPT_SGDM   g' = g + weight_decay*theta;  v <- momentum*v + g';  theta <- theta - eta_t*v   (state1 = v)
+ *   QSR_OPT_ADAMW  theta <- theta*(1 - eta_t*weight_decay);  m <- beta1*m + (1-beta1)*g;  v <- beta2*v + (1-beta2)*g^2;
+ *                  theta <- theta - eta_t * (m/(1-beta1^n)) / (sqrt(v)/sqrt(1-beta2^n) + eps)        (state1 = m, state2 = v)
+ *                  n = t + 1 - t_state_origin counts the steps the state has seen.
+ * Learning rate eta_t, t in {0..T-1} (Sec. 2): eta_max*t/T_warmup during warm-up, then, with
+ *   x = (t - T_warmup)/(T - T_warmup):  COSINE eta_min + (eta_max-eta_min)*(1+cos(pi*x))/2;  STEP_POW2 that value
+ *   rounded to 2^round(log2(.)) (Sec. 4, step-decay ablation);  LINEAR eta_min + (eta_max-eta_min)*(1-x);  CONST eta_max.
+ * Round length (Eq. 2): QSR_RULE_QSR H = max(H_base, floor((alpha/eta_t)^2)) with eta_t taken at the round's first
+ *   step, or at t = T_warmup for rounds that start during warm-up (Sec. 2); QSR_RULE_CONST_H H = H_base.  In both
+ *   cases H is cut to T - t so that the last round ends at T.
+ * Synthetic gradient (stands in for Sample() and back-propagation of Algorithm 2 when no gradient slab is
+ *   passed): g[k,i] = lambda[i]*(theta[k,i] - theta_star[i]) + noise_std*z(seed, worker_offset + k, t, i), where z is
+ *   a standard normal obtained by Box-Muller from Philox-4x32-10 with counter (i/4 low, i/4 high, t, worker) and
+ *   key = the two halves of seed; words (0,1) of the block serve i%4 in {0 (cos), 1 (sin)}, words (2,3) serve {2, 3};
+ *   each uniform is (top 23 bits + 1/2) / 2^23.
+ */
+typedef struct qsr_config {
+    int32_t K;              /* workers (rows) held in this process's slabs                                  */
+    int32_t worker_offset;  /* global index of row 0 (0 unless the workers are sharded over several GPUs)   */
+    int64_t P;              /* parameters per worker                                                        */
+    int64_t row_stride;     /* floats between consecutive rows                                              */
+    int32_t opt;            /* QSR_OPT_*                                                                    */
+    int32_t sched;          /* QSR_SCHED_*                                                                  */
+    int32_t rule;           /* QSR_RULE_*                                                                   */
+    int32_t state_sync;     /* QSR_STATE_*: what a synchronization does to state1/state2 (KEEP: nothing;   */
+                            /* AVERAGE: averaged like the parameters; RESET: zeroed, n restarts at 1)      */
+    double momentum, beta1, beta2, eps, weight_decay;
+    double eta_max, eta_min;
+    double alpha;           /* growth coefficient of Eq. 2                                                  */
+    double noise_std;
+    int64_t T, T_warmup, H_base;
+    int64_t t_state_origin; /* global step at which state1/state2 were last all-zero (0 for a fresh run)    */
+    uint64_t seed;
+} qsr_config;
+
+/* ---- host-only schedule (no device, no context) ------------------------------------------------------- */
+
+/* Validates the scalar fields (not the pointers).  QSR_OK, QSR_EINVAL, QSR_EALIGN or QSR_ERANGE. */
+int qsr_config_check(const qsr_config *cfg);
+
+/* eta_t in binary64 (Sec. 2; formulas above).  NaN if cfg is invalid or t is outside [0, T). */
+double qsr_config_learning_rate(const qsr_config *cfg, int64_t t);
+
+/* H of a round whose first global step is t (Eq. 2 with the warm-up and last-round rules).  Negative
+ * qsr_status on error. */
+int64_t qsr_config_round_length(const qsr_config *cfg, int64_t t);
+
+/* Writes the start step and the length of every round from t = 0 to T into round_start / round_len (host arrays
+ * of `cap` entries; entries beyond cap are counted but not written).  Returns the number of rounds, or a negative
+ * qsr_status.  The share of steps that synchronize (the "Comm." column of Tables 1-3) is rounds / T. */
+int64_t qsr_config_schedule(const qsr_config *cfg, int64_t *round_start, int64_t *round_len, int64_t cap);
+
+/* Bytes of device workspace that qsr_train_host needs for cfg (slabs plus the two input vectors). */
+int64_t qsr_workspace_bytes(const qsr_config *cfg);
+
+/* ---- context ------------------------------------------------------------------------------------------ */
+
+/* Creates a context over caller-owned slabs (Algorithm 2's workers).  params and state1 are [K, row_stride];
+ * state2 is required for QSR_OPT_ADAMW and ignored for QSR_OPT_SGDM; lambda and theta_star are [P] and may be NULL
+ * if every qsr_local_step will be given gradients.  cuda_stream is a cudaStream_t (NULL = the legacy default
+ * stream).  Nothing is written to the slabs.  The device current at this call is the one the context uses. */
+int qsr_init(qsr_ctx **out, const qsr_config *cfg, float *params, float *state1, float *state2,
+             const float *lambda, const float *theta_star, void *cuda_stream);
+
+/* Frees the context (host memory only).  NULL is accepted. */
+int qsr_destroy(qsr_ctx *ctx);
+
+/* Same as qsr_config_round_length on the context's configuration: GetH of Algorithm 2. */
+int64_t qsr_round_length(const qsr_ctx *ctx, int64_t t);
+
+/* theta[k, :] <- theta0_dev[0..P) for every worker k: "each worker gets a local copy of the global iterate"
+ * (Sec. 2).  Asynchronous. */
+int qsr_set_params(qsr_ctx *ctx, const float *theta0_dev);
+
+/* One local step of every worker at global iteration t (Eq. 1, inner loop of Algorithm 2), with learning rate
+ * eta_t and, for AdamW, bias corrections for n = t + 1 - t_state_origin, all evaluated on the host in binary64.
+ * grads == NULL: the gradient is generated inside the kernel (formula above) and never stored.
+ * grads != NULL: [K, row_stride] device slab read as the workers' gradients.  One kernel launch; asynchronous. */
+int qsr_local_step(qsr_ctx *ctx, int64_t t, const float *grads);
+
+/* End of a round (Algorithm 2): theta_bar[i] = (1/K) * sum_k theta[k,i], summed in fp32 for k = 0..K-1 and divided
+ * by K, then copied to every row; optimizer state treated per state_sync.  In RESET mode the bias-correction origin
+ * moves to t_next (the first step of the next round).  One kernel launch; asynchronous. */
+int qsr_sync(qsr_ctx *ctx, int64_t t_next);
+
+/* The same synchronization split in two for workers sharded over several GPUs: qsr_sync_partial writes
+ * sum[i] = sum_k theta[k,i] over this process's rows (and, in AVERAGE mode, the sums of state1 / state2 to
+ * sum + P and sum + 2P, each region rounded up to a multiple of 4 floats); the caller all-reduces `sum` over
+ * processes (SUM); qsr_sync_finish divides by K_total and writes every local row (and applies state_sync).
+ * `sum` holds qsr_sync_sum_floats(ctx) floats. */
+int64_t qsr_sync_sum_floats(const qsr_ctx *ctx);
+int qsr_sync_partial(qsr_ctx *ctx, float *sum);
+int qsr_sync_finish(qsr_ctx *ctx, const float *sum, int32_t K_total, int64_t t_next);
+
+/* Algorithm 2 from t_begin (which must be the first step of a round) until the first round end >= t_end
+ * (t_end <= T): per round GetH, H local steps with generated gradients, one synchronization.  The start and
+ * length of each round are written to the host arrays round_start / round_len (cap entries, may be NULL with
+ * cap = 0) and their count to *n_rounds (may be NULL).  Asynchronous: kernels are only enqueued. */
+int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
+            int64_t *round_start, int64_t *round_len, int64_t cap, int64_t *n_rounds);
+
+/* Kernel launches issued through this context so far. */
+int64_t qsr_launch_count(const qsr_ctx *ctx);
+
+/* Overrides the launch shape of the step kernel (threads per block: 64..1024, a multiple of 32; rows in flight
+ * per thread: 1, 2, 4 or 8) and of the sync kernel (threads per block: 64..512).  0 keeps the current value.  A
+ * step shape whose registers do not fit on an SM makes the next qsr_local_step return QSR_ECUDA. */
+int qsr_set_launch_shape(qsr_ctx *ctx, int32_t step_threads, int32_t step_rows_in_flight, int32_t sync_threads);
+
+/* ---- whole run from host memory ----------------------------------------------------------------------- */
+
+/* Algorithm 2 from theta_bar(0) to theta_bar(R) for callers whose data lives in host memory: copies
+ * theta0_host, lambda_host, theta_star_host ([P] each, pinned or pageable) to the device workspace, gives every
+ * worker a copy of theta0, zeroes the optimizer state, runs steps [0, t_end) as qsr_run does, copies worker 0's
+ * parameters (all workers are equal after the last synchronization) to theta_out_host [P], and waits for the
+ * stream.  workspace_dev: caller-owned device memory of at least qsr_workspace_bytes(cfg) bytes, 256-byte aligned.
+ * cfg->row_stride is ignored (rows are packed at P rounded up to 4).  round_* / n_rounds as in qsr_run;
+ * *launches (may be NULL) receives the number of kernel launches. */
+int qsr_train_host(const qsr_config *cfg, const float *theta0_host, const float *lambda_host,
+                   const float *theta_star_host, float *theta_out_host,
+                   void *workspace_dev, int64_t workspace_bytes, int64_t t_end, void *cuda_stream,
+                   int64_t *round_start, int64_t *round_len, int64_t cap, int64_t *n_rounds, int64_t *launches);
+
+/* Text for a qsr_status. Never NULL. */
+const char *qsr_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QSR_H_ */

@@ -1,0 +1,275 @@
+// C ABI of the library: argument checks, host-side scalars of each step, launches.  See include/qsr.h.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+
+struct qsr_ctx {
+    qsr_config cfg;
+    float *theta, *s1, *s2;
+    const float *lambda, *theta_star;
+    cudaStream_t stream;
+    qsr::LaunchShape shape;
+    int64_t t_state_origin;
+    int64_t launches;
+    bool partial_pending;
+};
+
+namespace {
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int64_t round_up4(int64_t n) { return (n + 3) & ~int64_t(3); }
+
+int n_state_slabs(const qsr_config &c) { return c.opt == QSR_OPT_ADAMW ? 2 : 1; }
+
+// Scalars of the local step at global iteration t (Eq. 1): everything that depends on t is evaluated here in
+// binary64 and rounded to fp32 once.
+qsr::StepParams step_params(const qsr_ctx &x, int64_t t, const float *grads)
+{
+    const qsr_config &c = x.cfg;
+    qsr::StepParams p;
+    std::memset(&p, 0, sizeof p);
+    p.theta = x.theta; p.s1 = x.s1; p.s2 = x.s2;
+    p.grads = grads; p.lambda = x.lambda; p.theta_star = x.theta_star;
+    p.P = c.P; p.stride = c.row_stride; p.K = c.K;
+    p.worker0 = uint32_t(c.worker_offset);
+    p.key0 = uint32_t(c.seed); p.key1 = uint32_t(c.seed >> 32);
+    p.step = uint32_t(t);
+    p.sigma = float(c.noise_std);
+    const double eta = qsr::learning_rate(c, t);
+    p.eta = float(eta); p.wd = float(c.weight_decay); p.mu = float(c.momentum);
+    const double n = double(t + 1 - x.t_state_origin);
+    const double bc1 = 1.0 - std::pow(c.beta1, n), bc2 = 1.0 - std::pow(c.beta2, n);
+    p.decay = float(1.0 - eta * c.weight_decay);
+    p.beta1 = float(c.beta1); p.beta2 = float(c.beta2);
+    p.omb1 = float(1.0 - c.beta1); p.omb2 = float(1.0 - c.beta2);
+    p.step_size = float(eta / bc1);
+    p.inv_sqrt_bc2 = float(1.0 / std::sqrt(bc2));
+    p.eps = float(c.eps);
+    return p;
+}
+
+qsr::SyncParams sync_params(const qsr_ctx &x)
+{
+    const qsr_config &c = x.cfg;
+    qsr::SyncParams p;
+    std::memset(&p, 0, sizeof p);
+    p.slab[0] = x.theta; p.slab[1] = x.s1; p.slab[2] = x.s2;
+    const int ns = n_state_slabs(c);
+    p.n_mean = c.state_sync == QSR_STATE_AVERAGE ? 1 + ns : 1;
+    p.n_zero = c.state_sync == QSR_STATE_RESET ? ns : 0;
+    p.P = c.P; p.stride = c.row_stride; p.K = c.K;
+    p.P4 = round_up4(c.P);
+    p.divisor = float(c.K);
+    return p;
+}
+
+int cuda_rc(int err) { return err == 0 ? QSR_OK : QSR_ECUDA; }
+
+}  // namespace
+
+extern "C" {
+
+int qsr_init(qsr_ctx **out, const qsr_config *cfg, float *params, float *state1, float *state2,
+             const float *lambda, const float *theta_star, void *cuda_stream)
+{
+    if (!out) return QSR_EINVAL;
+    *out = nullptr;
+    if (!cfg || !params || !state1) return QSR_EINVAL;
+    if (int rc = qsr::check_config(*cfg)) return rc;
+    if (cfg->opt == QSR_OPT_ADAMW && !state2) return QSR_EINVAL;
+    if ((lambda == nullptr) != (theta_star == nullptr)) return QSR_EINVAL;
+    if (!aligned16(params) || !aligned16(state1) || !aligned16(state2) || !aligned16(lambda) || !aligned16(theta_star))
+        return QSR_EALIGN;
+    if (int64_t(cfg->worker_offset) + cfg->K > (int64_t(1) << 32)) return QSR_ERANGE;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return QSR_ECUDA;
+    qsr_ctx *x = new (std::nothrow) qsr_ctx;
+    if (!x) return QSR_EINVAL;
+    x->cfg = *cfg;
+    x->theta = params; x->s1 = state1; x->s2 = cfg->opt == QSR_OPT_ADAMW ? state2 : nullptr;
+    x->lambda = lambda; x->theta_star = theta_star;
+    x->stream = static_cast<cudaStream_t>(cuda_stream);
+    x->shape = qsr::LaunchShape();
+    x->t_state_origin = cfg->t_state_origin;
+    x->launches = 0;
+    x->partial_pending = false;
+    *out = x;
+    return QSR_OK;
+}
+
+int qsr_destroy(qsr_ctx *ctx)
+{
+    delete ctx;
+    return QSR_OK;
+}
+
+int64_t qsr_round_length(const qsr_ctx *ctx, int64_t t)
+{
+    if (!ctx) return QSR_EINVAL;
+    if (t < 0 || t >= ctx->cfg.T) return QSR_ERANGE;
+    return qsr::round_length(ctx->cfg, t);
+}
+
+int qsr_set_params(qsr_ctx *ctx, const float *theta0_dev)
+{
+    if (!ctx || !theta0_dev) return QSR_EINVAL;
+    if (!aligned16(theta0_dev)) return QSR_EALIGN;
+    ctx->launches++;
+    return cuda_rc(qsr::launch_broadcast(ctx->theta, theta0_dev, ctx->cfg.P, ctx->cfg.row_stride, ctx->cfg.K,
+                                         ctx->shape, ctx->stream));
+}
+
+int qsr_local_step(qsr_ctx *ctx, int64_t t, const float *grads)
+{
+    if (!ctx) return QSR_EINVAL;
+    if (t < 0 || t >= ctx->cfg.T || t < ctx->t_state_origin) return QSR_ERANGE;
+    if (!grads && !ctx->lambda) return QSR_EINVAL;
+    if (!aligned16(grads)) return QSR_EALIGN;
+    const qsr::StepParams p = step_params(*ctx, t, grads);
+    ctx->launches++;
+    return cuda_rc(qsr::launch_step(p, ctx->cfg.opt, ctx->shape, ctx->stream));
+}
+
+int qsr_sync(qsr_ctx *ctx, int64_t t_next)
+{
+    if (!ctx) return QSR_EINVAL;
+    if (t_next < 0 || t_next > ctx->cfg.T) return QSR_ERANGE;
+    const qsr::SyncParams p = sync_params(*ctx);
+    ctx->launches++;
+    const int rc = cuda_rc(qsr::launch_sync(p, ctx->shape, ctx->stream));
+    if (rc == QSR_OK && ctx->cfg.state_sync == QSR_STATE_RESET) ctx->t_state_origin = t_next;
+    return rc;
+}
+
+int64_t qsr_sync_sum_floats(const qsr_ctx *ctx)
+{
+    if (!ctx) return QSR_EINVAL;
+    const int n_mean = ctx->cfg.state_sync == QSR_STATE_AVERAGE ? 1 + n_state_slabs(ctx->cfg) : 1;
+    return n_mean * round_up4(ctx->cfg.P);
+}
+
+int qsr_sync_partial(qsr_ctx *ctx, float *sum)
+{
+    if (!ctx || !sum) return QSR_EINVAL;
+    if (!aligned16(sum)) return QSR_EALIGN;
+    qsr::SyncParams p = sync_params(*ctx);
+    p.sum_out = sum;
+    ctx->launches++;
+    const int rc = cuda_rc(qsr::launch_sync_partial(p, ctx->shape, ctx->stream));
+    if (rc == QSR_OK) ctx->partial_pending = true;
+    return rc;
+}
+
+int qsr_sync_finish(qsr_ctx *ctx, const float *sum, int32_t K_total, int64_t t_next)
+{
+    if (!ctx || !sum) return QSR_EINVAL;
+    if (!aligned16(sum)) return QSR_EALIGN;
+    if (K_total < ctx->cfg.K || t_next < 0 || t_next > ctx->cfg.T) return QSR_ERANGE;
+    if (!ctx->partial_pending) return QSR_ESTATE;
+    qsr::SyncParams p = sync_params(*ctx);
+    p.sum_in = sum;
+    p.divisor = float(K_total);
+    ctx->launches++;
+    const int rc = cuda_rc(qsr::launch_sync_finish(p, ctx->shape, ctx->stream));
+    if (rc == QSR_OK) {
+        ctx->partial_pending = false;
+        if (ctx->cfg.state_sync == QSR_STATE_RESET) ctx->t_state_origin = t_next;
+    }
+    return rc;
+}
+
+int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
+            int64_t *round_start, int64_t *round_len, int64_t cap, int64_t *n_rounds)
+{
+    if (!ctx || cap < 0 || (cap > 0 && (!round_start || !round_len))) return QSR_EINVAL;
+    if (t_begin < 0 || t_end > ctx->cfg.T || t_begin > t_end) return QSR_ERANGE;
+    if (!ctx->lambda) return QSR_EINVAL;
+    int64_t s = 0;
+    for (int64_t t = t_begin; t < t_end;) {
+        const int64_t H = qsr::round_length(ctx->cfg, t);       // GetH
+        for (int64_t h = 0; h < H; ++h)
+            if (int rc = qsr_local_step(ctx, t + h, nullptr)) return rc;
+        if (int rc = qsr_sync(ctx, t + H)) return rc;           // parameter averaging
+        if (s < cap) {
+            round_start[s] = t;
+            round_len[s] = H;
+        }
+        ++s;
+        t += H;
+    }
+    if (n_rounds) *n_rounds = s;
+    return QSR_OK;
+}
+
+int64_t qsr_launch_count(const qsr_ctx *ctx) { return ctx ? ctx->launches : int64_t(QSR_EINVAL); }
+
+int qsr_set_launch_shape(qsr_ctx *ctx, int32_t step_threads, int32_t step_rows_in_flight, int32_t sync_threads)
+{
+    if (!ctx) return QSR_EINVAL;
+    auto ok_threads = [](int32_t n, int32_t hi) { return n == 0 || (n >= 64 && n <= hi && n % 32 == 0); };
+    if (!ok_threads(step_threads, 1024) || !ok_threads(sync_threads, 512)) return QSR_ERANGE;
+    if (step_rows_in_flight != 0 && step_rows_in_flight != 1 && step_rows_in_flight != 2 && step_rows_in_flight != 4 &&
+        step_rows_in_flight != 8)
+        return QSR_ERANGE;
+    if (step_threads) ctx->shape.step_threads = step_threads;
+    if (step_rows_in_flight) ctx->shape.step_rows = step_rows_in_flight;
+    if (sync_threads) ctx->shape.sync_threads = sync_threads;
+    return QSR_OK;
+}
+
+int64_t qsr_workspace_bytes(const qsr_config *cfg)
+{
+    if (!cfg) return QSR_EINVAL;
+    qsr_config c = *cfg;
+    c.row_stride = round_up4(c.P);
+    if (int rc = qsr::check_config(c)) return rc;
+    const int64_t slabs = 1 + n_state_slabs(c);
+    return (slabs * c.K * c.row_stride + 3 * c.row_stride) * int64_t(sizeof(float));
+}
+
+int qsr_train_host(const qsr_config *cfg, const float *theta0_host, const float *lambda_host,
+                   const float *theta_star_host, float *theta_out_host,
+                   void *workspace_dev, int64_t workspace_bytes, int64_t t_end, void *cuda_stream,
+                   int64_t *round_start, int64_t *round_len, int64_t cap, int64_t *n_rounds, int64_t *launches)
+{
+    if (!cfg || !theta0_host || !lambda_host || !theta_star_host || !theta_out_host || !workspace_dev) return QSR_EINVAL;
+    qsr_config c = *cfg;
+    c.row_stride = round_up4(c.P);
+    c.t_state_origin = 0;
+    if (int rc = qsr::check_config(c)) return rc;
+    if ((reinterpret_cast<uintptr_t>(workspace_dev) & 255u) != 0) return QSR_EALIGN;
+    const int64_t need = qsr_workspace_bytes(&c);
+    if (workspace_bytes < need || t_end < 0 || t_end > c.T) return QSR_ERANGE;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    float *w = static_cast<float *>(workspace_dev);
+    const int64_t slab = int64_t(c.K) * c.row_stride;
+    float *theta = w, *s1 = w + slab, *s2 = c.opt == QSR_OPT_ADAMW ? w + 2 * slab : nullptr;
+    float *vec = w + (1 + n_state_slabs(c)) * slab;
+    float *lambda = vec, *theta_star = vec + c.row_stride, *theta0 = vec + 2 * c.row_stride;
+    const size_t row_bytes = size_t(c.P) * sizeof(float);
+
+    if (cudaMemcpyAsync(lambda, lambda_host, row_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return QSR_ECUDA;
+    if (cudaMemcpyAsync(theta_star, theta_star_host, row_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return QSR_ECUDA;
+    if (cudaMemcpyAsync(theta0, theta0_host, row_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return QSR_ECUDA;
+    if (cudaMemsetAsync(s1, 0, size_t(n_state_slabs(c)) * slab * sizeof(float), st) != cudaSuccess) return QSR_ECUDA;
+
+    qsr_ctx *x = nullptr;
+    if (int rc = qsr_init(&x, &c, theta, s1, s2, lambda, theta_star, cuda_stream)) return rc;
+    int rc = qsr_set_params(x, theta0);
+    if (rc == QSR_OK) rc = qsr_run(x, 0, t_end, round_start, round_len, cap, n_rounds);
+    if (rc == QSR_OK && cudaMemcpyAsync(theta_out_host, theta, row_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        rc = QSR_ECUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess && rc == QSR_OK) rc = QSR_ECUDA;
+    if (launches) *launches = x->launches;
+    qsr_destroy(x);
+    return rc;
+}
+
+}  // extern "C"

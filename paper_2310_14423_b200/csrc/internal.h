@@ -1,0 +1,61 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#ifndef QSR_INTERNAL_H_
+#define QSR_INTERNAL_H_
+
+#include <cstdint>
+
+#include "../../include/qsr.h"
+
+namespace qsr {
+
+// schedule.cpp
+int check_config(const qsr_config &c);
+double learning_rate(const qsr_config &c, int64_t t);
+int64_t round_length(const qsr_config &c, int64_t t);
+
+// Arguments of one local-step launch.  Scalars are evaluated on the host in binary64 and rounded once.
+struct StepParams {
+    float *theta, *s1, *s2;
+    const float *grads;       // NULL: generate the gradient in the kernel
+    const float *lambda, *theta_star;
+    int64_t P, stride;
+    int32_t K;
+    uint32_t worker0;         // global index of row 0
+    uint32_t key0, key1;      // Philox key (seed halves)
+    uint32_t step;            // global iteration t (Philox counter word 2)
+    float sigma;              // noise_std
+    float eta, wd, mu;        // SGD with momentum
+    float decay;              // AdamW: 1 - eta*wd
+    float beta1, beta2, omb1, omb2;
+    float step_size;          // AdamW: eta / (1 - beta1^n)
+    float inv_sqrt_bc2;       // AdamW: 1 / sqrt(1 - beta2^n)
+    float eps;
+};
+
+struct SyncParams {
+    float *slab[3];           // arrays to average (theta first), then arrays to zero
+    int32_t n_mean, n_zero;
+    int64_t P, stride;
+    int32_t K;
+    float *sum_out;           // partial mode: per-array sums, array a at sum_out + a*P4
+    const float *sum_in;      // finish mode: all-reduced sums
+    int64_t P4;               // P rounded up to a multiple of 4
+    float divisor;            // K (or the global worker count in finish mode)
+};
+
+struct LaunchShape {
+    int step_threads = 256;
+    int step_rows = 2;
+    int sync_threads = 256;
+};
+
+// kernels.cu -- each returns a cudaError_t cast to int (0 = success) after enqueueing one kernel.
+int launch_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream);
+int launch_sync(const SyncParams &p, const LaunchShape &shape, void *stream);          // mean + write back (+ zero)
+int launch_sync_partial(const SyncParams &p, const LaunchShape &shape, void *stream);  // sums only
+int launch_sync_finish(const SyncParams &p, const LaunchShape &shape, void *stream);   // sums -> rows (+ zero)
+int launch_broadcast(float *theta, const float *theta0, int64_t P, int64_t stride, int32_t K,
+                     const LaunchShape &shape, void *stream);
+
+}  // namespace qsr
+#endif

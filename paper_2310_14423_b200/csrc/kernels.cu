@@ -1,0 +1,310 @@
+// CUDA kernels of the Local-OPT hot path for sm_100a: the fused local step (Eq. 1 of arXiv 2310.14423, with the
+// synthetic gradient generated in registers) and the replica-axis mean that ends a round (Algorithm 2).
+//
+// Both are pure HBM streams over [K, P] fp32 slabs: nothing here is a contraction, so there are no tensor-core
+// instructions.  A thread owns one 16-byte column (4 consecutive coordinates) for ALL K rows: lambda / theta_star
+// are fetched once per column instead of once per worker, every global access is a 128-bit LDG/STG on a
+// 16-byte boundary, a warp touches 512 contiguous bytes per row, and the loads of several rows are issued before
+// the first use so that each SM keeps enough bytes in flight to cover HBM latency.
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "internal.h"
+
+namespace qsr {
+namespace {
+
+// ---------------------------------------------------------------------------------------------- noise
+
+// Philox-4x32 with 10 rounds (Salmon et al., SC'11): 128-bit counter, 64-bit key.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1)
+{
+    constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(M0, c.x), lo0 = M0 * c.x;
+        const uint32_t hi1 = __umulhi(M1, c.z), lo1 = M1 * c.z;
+        c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+        k0 += W0;
+        k1 += W1;
+    }
+    return c;
+}
+
+// Box-Muller on two words: uniforms are (top 23 bits + 1/2) / 2^23, exact in fp32 and never 0 or 1.
+__device__ __forceinline__ void box_muller(uint32_t wa, uint32_t wb, float &z_cos, float &z_sin)
+{
+    const float u1 = (float(wa >> 9) + 0.5f) * 0x1p-23f;
+    const float two_u2 = (float(wb >> 9) + 0.5f) * 0x1p-22f;  // angle / pi
+    const float radius = sqrtf(-2.0f * logf(u1));
+    float s, c;
+    sincospif(two_u2, &s, &c);
+    z_cos = radius * c;
+    z_sin = radius * s;
+}
+
+// Four standard normals for coordinates 4j .. 4j+3 of one worker at one step.
+__device__ __forceinline__ float4 noise4(int64_t j, uint32_t step, uint32_t worker, uint32_t key0, uint32_t key1)
+{
+    const uint4 r = philox4x32_10(make_uint4(uint32_t(j), uint32_t(uint64_t(j) >> 32), step, worker), key0, key1);
+    float4 z;
+    box_muller(r.x, r.y, z.x, z.y);
+    box_muller(r.z, r.w, z.z, z.w);
+    return z;
+}
+
+// ---------------------------------------------------------------------------------------------- OPT (Eq. 1)
+
+template <int OPT>
+__device__ __forceinline__ void opt_update(float &theta, float &a, float &b, float g, const StepParams &p)
+{
+    if (OPT == QSR_OPT_SGDM) {
+        g = fmaf(p.wd, theta, g);          // L2 weight decay enters the gradient
+        a = fmaf(p.mu, a, g);              // heavy-ball buffer
+        theta = fmaf(-p.eta, a, theta);
+    } else {
+        theta *= p.decay;                  // decoupled weight decay
+        a = fmaf(p.beta1, a, p.omb1 * g);
+        b = fmaf(p.beta2, b, p.omb2 * g * g);
+        const float denom = fmaf(sqrtf(b), p.inv_sqrt_bc2, p.eps);
+        theta = fmaf(-p.step_size, a / denom, theta);
+    }
+}
+
+__device__ __forceinline__ float4 ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ void st4(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }
+
+// No launch bound: the register count decides how many threads fit; a block shape that does not fit is
+// reported by the launch as an error, not silently spilled.
+template <int OPT, bool EXT_GRAD, int ROWS>
+__global__ void local_step_kernel(const StepParams p)
+{
+    const int64_t n_col = (p.P + 3) >> 2;
+    const int64_t grid_stride = int64_t(gridDim.x) * blockDim.x;
+    for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < n_col; j += grid_stride) {
+        const int64_t i0 = j << 2;
+        if (i0 + 4 <= p.P) {
+            float4 lam = make_float4(0.f, 0.f, 0.f, 0.f), ths = lam;
+            if (!EXT_GRAD) {
+                lam = ld4(p.lambda + i0);
+                ths = ld4(p.theta_star + i0);
+            }
+            for (int k = 0; k < p.K; k += ROWS) {
+                float4 th[ROWS], a[ROWS], b[ROWS], g[ROWS];
+#pragma unroll
+                for (int r = 0; r < ROWS; ++r) {
+                    if (k + r < p.K) {
+                        const int64_t e = int64_t(k + r) * p.stride + i0;
+                        th[r] = ld4(p.theta + e);
+                        a[r] = ld4(p.s1 + e);
+                        if (OPT == QSR_OPT_ADAMW) b[r] = ld4(p.s2 + e);
+                        if (EXT_GRAD) g[r] = ld4(p.grads + e);
+                    }
+                }
+#pragma unroll
+                for (int r = 0; r < ROWS; ++r) {
+                    if (k + r < p.K) {
+                        const int64_t e = int64_t(k + r) * p.stride + i0;
+                        if (!EXT_GRAD) {
+                            const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k + r), p.key0, p.key1);
+                            g[r].x = fmaf(p.sigma, z.x, lam.x * (th[r].x - ths.x));
+                            g[r].y = fmaf(p.sigma, z.y, lam.y * (th[r].y - ths.y));
+                            g[r].z = fmaf(p.sigma, z.z, lam.z * (th[r].z - ths.z));
+                            g[r].w = fmaf(p.sigma, z.w, lam.w * (th[r].w - ths.w));
+                        }
+                        opt_update<OPT>(th[r].x, a[r].x, b[r].x, g[r].x, p);
+                        opt_update<OPT>(th[r].y, a[r].y, b[r].y, g[r].y, p);
+                        opt_update<OPT>(th[r].z, a[r].z, b[r].z, g[r].z, p);
+                        opt_update<OPT>(th[r].w, a[r].w, b[r].w, g[r].w, p);
+                        st4(p.theta + e, th[r]);
+                        st4(p.s1 + e, a[r]);
+                        if (OPT == QSR_OPT_ADAMW) st4(p.s2 + e, b[r]);
+                    }
+                }
+            }
+        } else {
+            // Ragged last column: P is not a multiple of 4.  Scalar accesses, nothing beyond P is touched.
+            const int valid = int(p.P - i0);
+            for (int k = 0; k < p.K; ++k) {
+                float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (!EXT_GRAD) z = noise4(j, p.step, p.worker0 + uint32_t(k), p.key0, p.key1);
+                for (int c = 0; c < valid; ++c) {
+                    const int64_t e = int64_t(k) * p.stride + i0 + c;
+                    float th = p.theta[e], a = p.s1[e], b = OPT == QSR_OPT_ADAMW ? p.s2[e] : 0.f;
+                    const float zc = c == 0 ? z.x : (c == 1 ? z.y : z.z);   // valid <= 3
+                    const float g = EXT_GRAD ? p.grads[e]
+                                             : fmaf(p.sigma, zc, p.lambda[i0 + c] * (th - p.theta_star[i0 + c]));
+                    opt_update<OPT>(th, a, b, g, p);
+                    p.theta[e] = th;
+                    p.s1[e] = a;
+                    if (OPT == QSR_OPT_ADAMW) p.s2[e] = b;
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------- synchronization
+
+__device__ __forceinline__ float4 add4(float4 x, float4 y) { return make_float4(x.x + y.x, x.y + y.y, x.z + y.z, x.w + y.w); }
+__device__ __forceinline__ float4 div4(float4 x, float d) { return make_float4(x.x / d, x.y / d, x.z / d, x.w / d); }
+
+// Sum over rows of one 16-byte column, k ascending, eight loads in flight.
+__device__ __forceinline__ float4 column_sum(const float *slab, int64_t i0, int64_t stride, int K)
+{
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    int k = 0;
+    for (; k + 8 <= K; k += 8) {
+        float4 v[8];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) v[r] = ld4(slab + int64_t(k + r) * stride + i0);
+#pragma unroll
+        for (int r = 0; r < 8; ++r) acc = add4(acc, v[r]);
+    }
+    for (; k < K; ++k) acc = add4(acc, ld4(slab + int64_t(k) * stride + i0));
+    return acc;
+}
+
+// One array's share of a synchronization for the column (or ragged tail) that starts at coordinate i0.
+// MODE 0: mean of the rows, written back to every row (the whole synchronization on one GPU).
+// MODE 1: sums only, written to sum_out (first half of a synchronization sharded over GPUs).
+// MODE 2: rows <- sum_in / divisor (second half).
+template <int MODE>
+__device__ __forceinline__ void sync_column(float *slab, const float *sum_in, float *sum_out, int64_t i0,
+                                            const SyncParams &p)
+{
+    if (i0 + 4 <= p.P) {
+        float4 s;
+        if (MODE == 2) s = ld4(sum_in + i0);
+        else s = column_sum(slab, i0, p.stride, p.K);
+        if (MODE == 1) {
+            st4(sum_out + i0, s);
+        } else {
+            const float4 mean = div4(s, p.divisor);
+#pragma unroll 4
+            for (int k = 0; k < p.K; ++k) st4(slab + int64_t(k) * p.stride + i0, mean);
+        }
+    } else {
+        for (int64_t i = i0; i < p.P; ++i) {
+            float s = 0.f;
+            if (MODE == 2) s = sum_in[i];
+            else for (int k = 0; k < p.K; ++k) s += slab[int64_t(k) * p.stride + i];
+            if (MODE == 1) {
+                sum_out[i] = s;
+            } else {
+                const float mean = s / p.divisor;
+                for (int k = 0; k < p.K; ++k) slab[int64_t(k) * p.stride + i] = mean;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void zero_column(float *slab, int64_t i0, const SyncParams &p)
+{
+    if (i0 + 4 <= p.P) {
+        const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+        for (int k = 0; k < p.K; ++k) st4(slab + int64_t(k) * p.stride + i0, zero);
+    } else {
+        for (int64_t i = i0; i < p.P; ++i)
+            for (int k = 0; k < p.K; ++k) slab[int64_t(k) * p.stride + i] = 0.f;
+    }
+}
+
+// slab[0 .. n_mean) are averaged (theta always; the optimizer state in AVERAGE mode); in modes 0 and 2 the
+// arrays slab[n_mean .. n_mean+n_zero) are zero-filled (state reset).
+template <int MODE>
+__global__ void __launch_bounds__(512) sync_kernel(const SyncParams p)
+{
+    const int64_t n_col = (p.P + 3) >> 2;
+    const int64_t grid_stride = int64_t(gridDim.x) * blockDim.x;
+    for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < n_col; j += grid_stride) {
+        const int64_t i0 = j << 2;
+#pragma unroll
+        for (int a = 0; a < 3; ++a) {
+            if (a < p.n_mean)
+                sync_column<MODE>(p.slab[a], p.sum_in + a * p.P4, p.sum_out + a * p.P4, i0, p);
+            else if (MODE != 1 && a < p.n_mean + p.n_zero)
+                zero_column(p.slab[a], i0, p);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(512) broadcast_kernel(float *theta, const float *theta0, int64_t P, int64_t stride, int K)
+{
+    const int64_t n_col = (P + 3) >> 2;
+    const int64_t grid_stride = int64_t(gridDim.x) * blockDim.x;
+    for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < n_col; j += grid_stride) {
+        const int64_t i0 = j << 2;
+        if (i0 + 4 <= P) {
+            const float4 v = ld4(theta0 + i0);
+            for (int k = 0; k < K; ++k) st4(theta + int64_t(k) * stride + i0, v);
+        } else {
+            for (int64_t i = i0; i < P; ++i)
+                for (int k = 0; k < K; ++k) theta[int64_t(k) * stride + i] = theta0[i];
+        }
+    }
+}
+
+unsigned grid_for(int64_t P, int threads)
+{
+    const int64_t n_col = (P + 3) >> 2;
+    int64_t blocks = (n_col + threads - 1) / threads;
+    const int64_t cap = 1 << 30;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return unsigned(blocks);
+}
+
+template <int OPT, bool EXT>
+int launch_step_rows(const StepParams &p, const LaunchShape &s, cudaStream_t st)
+{
+    const unsigned grid = grid_for(p.P, s.step_threads);
+    switch (s.step_rows) {
+    case 1: local_step_kernel<OPT, EXT, 1><<<grid, s.step_threads, 0, st>>>(p); break;
+    case 2: local_step_kernel<OPT, EXT, 2><<<grid, s.step_threads, 0, st>>>(p); break;
+    case 4: local_step_kernel<OPT, EXT, 4><<<grid, s.step_threads, 0, st>>>(p); break;
+    default: local_step_kernel<OPT, EXT, 8><<<grid, s.step_threads, 0, st>>>(p); break;
+    }
+    return int(cudaGetLastError());
+}
+
+}  // namespace
+
+int launch_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool ext = p.grads != nullptr;
+    if (opt == QSR_OPT_SGDM)
+        return ext ? launch_step_rows<QSR_OPT_SGDM, true>(p, shape, st) : launch_step_rows<QSR_OPT_SGDM, false>(p, shape, st);
+    return ext ? launch_step_rows<QSR_OPT_ADAMW, true>(p, shape, st) : launch_step_rows<QSR_OPT_ADAMW, false>(p, shape, st);
+}
+
+int launch_sync(const SyncParams &p, const LaunchShape &shape, void *stream)
+{
+    sync_kernel<0><<<grid_for(p.P, shape.sync_threads), shape.sync_threads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return int(cudaGetLastError());
+}
+
+int launch_sync_partial(const SyncParams &p, const LaunchShape &shape, void *stream)
+{
+    sync_kernel<1><<<grid_for(p.P, shape.sync_threads), shape.sync_threads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return int(cudaGetLastError());
+}
+
+int launch_sync_finish(const SyncParams &p, const LaunchShape &shape, void *stream)
+{
+    sync_kernel<2><<<grid_for(p.P, shape.sync_threads), shape.sync_threads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return int(cudaGetLastError());
+}
+
+int launch_broadcast(float *theta, const float *theta0, int64_t P, int64_t stride, int32_t K,
+                     const LaunchShape &shape, void *stream)
+{
+    broadcast_kernel<<<grid_for(P, shape.sync_threads), shape.sync_threads, 0, static_cast<cudaStream_t>(stream)>>>(
+        theta, theta0, P, stride, K);
+    return int(cudaGetLastError());
+}
+
+}  // namespace qsr

@@ -1,0 +1,170 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol the header declares, validates its
+arguments, and its host schedule (learning rate, round lengths) equals the oracle's bit for bit.
+No device work is issued here."""
+import ctypes as C
+import math
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import qsr_oracle as O
+from paper_2310_14423_b200 import binding as B
+from paper_2310_14423_b200 import build as qsr_build
+from paper_2310_14423_b200 import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+IMAGENET_TRAIN = 1_281_167
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    qsr_build.build()
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "qsr.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(qsr_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    declared = _declared_functions()
+    assert len(declared) >= 15
+    raw = C.CDLL(B.LIB_PATH)
+    for name in declared:
+        assert hasattr(raw, name), name
+    assert sorted(B.EXPORTS) == declared
+
+
+def test_config_struct_matches_header_size():
+    # 4 int32 + 2 int64 interleaved as in the header, 9 doubles, 4 int64, 1 uint64: 8 + 16 + 16 + 72 + 32 + 8
+    assert C.sizeof(B.QsrConfig) == 152
+
+
+def test_strerror_and_status_codes():
+    assert B.strerror(0) == "ok"
+    for code in (-1, -2, -3, -4, -5, -99):
+        assert B.strerror(code)
+
+
+def test_config_validation():
+    w = W.workload("c1")
+    ok = B.make_config(w)
+    assert B.qsr_config_check(ok) == B.QSR_OK
+
+    def bad(**kw):
+        c = B.make_config(w)
+        for k, v in kw.items():
+            setattr(c, k, v)
+        return B.qsr_config_check(c)
+
+    assert bad(K=0) == B.QSR_EINVAL
+    assert bad(P=0) == B.QSR_EINVAL
+    assert bad(opt=7) == B.QSR_EINVAL
+    assert bad(sched=-1) == B.QSR_EINVAL
+    assert bad(rule=2) == B.QSR_EINVAL
+    assert bad(state_sync=3) == B.QSR_EINVAL
+    assert bad(eta_max=float("nan")) == B.QSR_EINVAL
+    assert bad(alpha=float("inf")) == B.QSR_EINVAL
+    assert bad(eta_max=-0.1) == B.QSR_EINVAL
+    assert bad(row_stride=65538) == B.QSR_EALIGN
+    assert bad(row_stride=65532) == B.QSR_EALIGN
+    assert bad(T=0) == B.QSR_ERANGE
+    assert bad(T_warmup=2000) == B.QSR_ERANGE
+    assert bad(H_base=0) == B.QSR_ERANGE
+    assert bad(T=(1 << 32) + 1) == B.QSR_ERANGE
+    assert math.isnan(B.qsr_config_learning_rate(ok, -1))
+    assert math.isnan(B.qsr_config_learning_rate(ok, 2000))
+    with pytest.raises(B.QsrError) as e:
+        B.qsr_config_round_length(ok, 2000)
+    assert e.value.status == B.QSR_ERANGE
+    assert B.lib().qsr_config_round_length(None, 0) == B.QSR_EINVAL
+    assert B.lib().qsr_round_length(None, 0) == B.QSR_EINVAL
+    assert B.lib().qsr_local_step(None, 0, None) == B.QSR_EINVAL
+    assert B.lib().qsr_sync(None, 0) == B.QSR_EINVAL
+    assert B.lib().qsr_destroy(None) == B.QSR_OK
+
+
+def test_init_rejects_bad_pointers_without_touching_a_device():
+    cfg = B.make_config(W.workload("c2"))
+    h = C.c_void_p()
+    L = B.lib()
+    assert L.qsr_init(None, C.byref(cfg), 256, 256, 256, 256, 256, None) == B.QSR_EINVAL
+    assert L.qsr_init(C.byref(h), None, 256, 256, 256, 256, 256, None) == B.QSR_EINVAL
+    assert L.qsr_init(C.byref(h), C.byref(cfg), None, 256, 256, 256, 256, None) == B.QSR_EINVAL
+    assert L.qsr_init(C.byref(h), C.byref(cfg), 256, 256, None, 256, 256, None) == B.QSR_EINVAL   # AdamW needs state2
+    assert L.qsr_init(C.byref(h), C.byref(cfg), 256, 256, 256, 256, None, None) == B.QSR_EINVAL   # lambda without theta*
+    assert L.qsr_init(C.byref(h), C.byref(cfg), 260, 256, 256, 256, 256, None) == B.QSR_EALIGN
+    assert L.qsr_init(C.byref(h), C.byref(cfg), 256, 256, 256, 264, 256, None) == B.QSR_EALIGN
+    assert not h.value
+
+
+def test_workspace_bytes():
+    w = W.workload("c2")
+    cfg = B.make_config(w)
+    assert B.qsr_workspace_bytes(cfg) == (3 * w.K * w.P + 3 * w.P) * 4
+    w = W.tiny_workload(W.OPT_SGDM, K=3, P=1001)
+    assert B.qsr_workspace_bytes(B.make_config(w)) == (2 * 3 * 1004 + 3 * 1004) * 4
+
+
+def _same_schedule(w):
+    cfg = B.make_config(w)
+    st, H = B.qsr_config_schedule(cfg)
+    ost, oH = O.schedule(w)
+    assert np.array_equal(st, ost) and np.array_equal(H, oH)
+    return st, H
+
+
+def test_schedule_equals_oracle_on_the_run_configurations():
+    for name in ("c1", "c2", "c3", "c4", "c4p", "c5"):
+        w = W.workload(name)
+        st, H = _same_schedule(w)
+        for sched in (W.SCHED_STEP_POW2, W.SCHED_LINEAR, W.SCHED_CONST):
+            _same_schedule(w.replace(sched=sched))
+        _same_schedule(w.replace(eta_min=1e-6))
+    # the sweep: growth coefficients x minimum periods, and constant periods, at both peak learning rates
+    for eta_max in (8e-4, 8e-3):
+        for alpha in (0.01, 0.0175, 0.025):
+            for Hb in (2, 4, 8):
+                _same_schedule(W.workload("c5").replace(eta_max=eta_max, alpha=alpha, H_base=Hb))
+    for Hb in (2, 4, 8):
+        _same_schedule(W.workload("c5").replace(rule=W.RULE_CONST_H, H_base=Hb))
+
+
+def test_schedule_equals_oracle_on_the_papers_runs(golden_dir):
+    """The 13 runs of Tables 1-3 / the linear-decay figure: same rounds as the oracle, hence the printed volumes."""
+    n = 0
+    with open(os.path.join(golden_dir, "paper_comm_volumes.txt")) as f:
+        for line in f:
+            if not line.strip() or line.startswith("#"):
+                continue
+            label, model, sched, batch, epochs, warm, eta_max, alpha, Hb, comm, src = line.split()
+            per_epoch = IMAGENET_TRAIN // int(batch)
+            T = int(epochs) * per_epoch
+            T_w = int(warm[:-2]) * per_epoch if warm.endswith("ep") else int(warm[:-2])
+            w = W.Workload(label, 1, W.flat_layout(4), W.OPT_SGDM, T=T, T_warmup=T_w, eta_max=float(eta_max),
+                           sched=sched, alpha=float(alpha), H_base=int(Hb))
+            st, H = _same_schedule(w)
+            assert abs(100.0 * len(st) / T - float(comm)) <= 0.055
+            n += 1
+    assert n == 13
+
+
+def test_learning_rate_equals_oracle_bitwise():
+    for name in ("c1", "c2", "c4"):
+        for sched in (W.SCHED_COSINE, W.SCHED_STEP_POW2, W.SCHED_LINEAR, W.SCHED_CONST):
+            w = W.workload(name).replace(sched=sched)
+            cfg = B.make_config(w)
+            for t in list(range(0, w.T, 97)) + [w.T - 1, w.T_warmup, max(0, w.T_warmup - 1)]:
+                assert B.qsr_config_learning_rate(cfg, t) == O.lr(w, t), (name, sched, t)
+
+
+def test_round_length_pointwise_and_truncation():
+    w = W.workload("c1")
+    cfg = B.make_config(w)
+    for t in range(0, w.T, 13):
+        assert B.qsr_config_round_length(cfg, t) == O.round_length(w, t)
+    assert B.qsr_config_round_length(cfg, 1999) == 1
+    assert B.qsr_config_round_length(cfg, 0) == 4          # (0.2/0.1)^2 is exactly 4 in binary64
