@@ -45,7 +45,7 @@ qsr::StepParams step_params(const qsr_ctx &x, int64_t t, const float *grads)
     p.eta = float(eta); p.wd = float(c.weight_decay); p.mu = float(c.momentum);
     const double n = double(t + 1 - x.t_state_origin);
     const double bc1 = 1.0 - std::pow(c.beta1, n), bc2 = 1.0 - std::pow(c.beta2, n);
-    p.decay = float(1.0 - eta * c.weight_decay);
+    p.eta_wd = float(eta * c.weight_decay);
     p.beta1 = float(c.beta1); p.beta2 = float(c.beta2);
     p.omb1 = float(1.0 - c.beta1); p.omb2 = float(1.0 - c.beta2);
     p.step_size = float(eta / bc1);

@@ -25,7 +25,7 @@ struct StepParams {
     uint32_t step;            // global iteration t (Philox counter word 2)
     float sigma;              // noise_std
     float eta, wd, mu;        // SGD with momentum
-    float decay;              // AdamW: 1 - eta*wd
+    float eta_wd;             // AdamW: eta * weight_decay
     float beta1, beta2, omb1, omb2;
     float step_size;          // AdamW: eta / (1 - beta1^n)
     float inv_sqrt_bc2;       // AdamW: 1 / sqrt(1 - beta2^n)

@@ -64,11 +64,14 @@ __device__ __forceinline__ void opt_update(float &theta, float &a, float &b, flo
         a = fmaf(p.mu, a, g);              // heavy-ball buffer
         theta = fmaf(-p.eta, a, theta);
     } else {
-        theta *= p.decay;                  // decoupled weight decay
         a = fmaf(p.beta1, a, p.omb1 * g);
         b = fmaf(p.beta2, b, p.omb2 * g * g);
         const float denom = fmaf(sqrtf(b), p.inv_sqrt_bc2, p.eps);
-        theta = fmaf(-p.step_size, a / denom, theta);
+        // theta*(1 - eta*wd) - step_size*m/denom as ONE subtraction from theta.  Forming 1 - eta*wd in fp32 would
+        // keep only ~2^-24 of absolute precision on a term of size eta*wd, and the product theta*(1 - eta*wd) has
+        // near-ties that round the same way step after step when theta sits just above a power of two; both show up
+        // as a drift of a few 1e-5 over thousands of small steps.  The decay and the update are summed first instead.
+        theta -= fmaf(p.eta_wd, theta, p.step_size * (a / denom));
     }
 }
 

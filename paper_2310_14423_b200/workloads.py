@@ -185,6 +185,10 @@ def workload(name: str) -> Workload:
     c4p as c4 with the paper's peak lr 0.008 (App. C.2), so that H_base shapes the schedule
     c5  K=32, ViT-B/16 shapes (sweep base: alpha, H_base and the rule are overridden by the caller)
     """
+    if name in ("c3s", "c4s", "c4ps"):
+        # The same runs on a flat 2^23-parameter set: slabs of 512 MiB, larger than L2 but small enough for
+        # profiler captures that replay each launch many times.
+        return workload(name[:-1]).replace(name=name, layout=flat_layout(1 << 23))
     if name == "c1":
         return Workload("c1", 4, flat_layout(65536), OPT_SGDM, T=2000, T_warmup=0, eta_max=0.1,
                         alpha=0.2, H_base=2, momentum=0.9, noise_std=0.1,
