@@ -142,6 +142,31 @@ int64_t qsr_sync_sum_floats(const qsr_ctx *ctx);
 int qsr_sync_partial(qsr_ctx *ctx, float *sum);
 int qsr_sync_finish(qsr_ctx *ctx, const float *sum, int32_t K_total, int64_t t_next);
 
+/* A synchronization for callers that have no device buffer to spare and may not create one.  The paper has no
+ * counterpart to this call: it exists for the way this library gets used.  Some hosts of this code run inside a
+ * process whose device memory is handed out once, up front, by another component (a serving runtime, a framework's
+ * caching allocator with a hard budget, a job that has already filled the GPU with its slabs), and some call from
+ * places where cudaMalloc is not welcome because it stalls the whole device or is simply not permitted there.
+ * Such callers cannot provide the `sum` buffer that qsr_sync_partial / qsr_sync_finish need.
+ *
+ * qsr_sync_static does the same two phases -- row sums, then rows <- sums / K (and the state_sync treatment) --
+ * through a fixed array of QSR_STATIC_SCRATCH_FLOATS floats that is part of the library image, so every GPU that
+ * loads the library holds that much memory until the process exits.  The call allocates and frees nothing.  The
+ * result equals qsr_sync's: the same fp32 sum over k = 0..K-1 and the same single division by K.
+ *
+ * Limits and rules
+ *   - The sums must fit: (P rounded up to 4) floats, times 1 + the number of state slabs in AVERAGE mode, must not
+ *     exceed QSR_STATIC_SCRATCH_FLOATS.  Larger problems get QSR_ERANGE and nothing is launched; use qsr_sync, or
+ *     qsr_sync_partial / qsr_sync_finish with a buffer of your own.
+ *   - The first call on a device looks up the array's device address (once per device; the context's device must be
+ *     current, as for every call).  Make that first call before any stream capture begins.
+ *   - All contexts and all calls in the process share the one array.  Each call overwrites what it needs before
+ *     reading it, so an earlier call's leftovers are harmless; but two calls whose kernels can overlap on the GPU
+ *     (different streams, no ordering between them) race on it.  Keep the calls on one stream or order them.
+ * Two kernel launches; asynchronous. */
+#define QSR_STATIC_SCRATCH_FLOATS (1 << 20) /* 4 MiB */
+int qsr_sync_static(qsr_ctx *ctx, int64_t t_next);
+
 /* Algorithm 2 from t_begin (which must be the first step of a round) until the first round end >= t_end
  * (t_end <= T): per round GetH, H local steps with generated gradients, one synchronization.  The start and
  * length of each round are written to the host arrays round_start / round_len (cap entries, may be NULL with

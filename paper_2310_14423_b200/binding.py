@@ -23,10 +23,11 @@ RULE = {"qsr": 0, "const_h": 1}
 STATE = {"keep": 0, "average": 1, "reset": 2}
 
 QSR_OK, QSR_EINVAL, QSR_EALIGN, QSR_ECUDA, QSR_ERANGE, QSR_ESTATE = 0, -1, -2, -3, -4, -5
+QSR_STATIC_SCRATCH_FLOATS = 1 << 20
 
 EXPORTS = ("qsr_config_check", "qsr_config_learning_rate", "qsr_config_round_length", "qsr_config_schedule",
            "qsr_workspace_bytes", "qsr_init", "qsr_destroy", "qsr_round_length", "qsr_set_params", "qsr_local_step",
-           "qsr_sync", "qsr_sync_sum_floats", "qsr_sync_partial", "qsr_sync_finish", "qsr_run", "qsr_launch_count",
+           "qsr_sync", "qsr_sync_sum_floats", "qsr_sync_partial", "qsr_sync_finish", "qsr_sync_static", "qsr_run", "qsr_launch_count",
            "qsr_set_launch_shape", "qsr_train_host", "qsr_strerror")
 
 
@@ -74,6 +75,7 @@ def lib():
             "qsr_sync_sum_floats": (i64, [vp]),
             "qsr_sync_partial": (C.c_int, [vp, vp]),
             "qsr_sync_finish": (C.c_int, [vp, vp, i32, i64]),
+            "qsr_sync_static": (C.c_int, [vp, i64]),
             "qsr_run": (C.c_int, [vp, i64, i64, vp, vp, i64, C.POINTER(i64)]),
             "qsr_launch_count": (i64, [vp]),
             "qsr_set_launch_shape": (C.c_int, [vp, i32, i32, i32]),
@@ -198,6 +200,11 @@ class Context:
 
     def qsr_sync_finish(self, sums, K_total: int, t_next: int) -> None:
         _check(lib().qsr_sync_finish(self._h, _dptr(sums), int(K_total), int(t_next)), "qsr_sync_finish")
+
+    def qsr_sync_static(self, t_next: int) -> None:
+        """qsr_sync through the library's built-in scratch array: for callers that cannot allocate the `sum` buffer.
+        Raises QsrError(QSR_ERANGE) when the problem exceeds QSR_STATIC_SCRATCH_FLOATS."""
+        _check(lib().qsr_sync_static(self._h, int(t_next)), "qsr_sync_static")
 
     def qsr_run(self, t_begin: int = 0, t_end: Optional[int] = None) -> Tuple[np.ndarray, np.ndarray]:
         t_end = int(self.cfg.T if t_end is None else t_end)

@@ -184,6 +184,19 @@ int qsr_sync_finish(qsr_ctx *ctx, const float *sum, int32_t K_total, int64_t t_n
     return rc;
 }
 
+int qsr_sync_static(qsr_ctx *ctx, int64_t t_next)
+{
+    if (!ctx) return QSR_EINVAL;
+    if (t_next < 0 || t_next > ctx->cfg.T) return QSR_ERANGE;
+    const qsr::SyncParams p = sync_params(*ctx);
+    if (int64_t(p.n_mean) * p.P4 > int64_t(QSR_STATIC_SCRATCH_FLOATS)) return QSR_ERANGE;   // nothing was launched
+    const int err = qsr::launch_sync_static(p, ctx->shape, ctx->stream);
+    if (err != 0) return err == -1 ? QSR_ERANGE : QSR_ECUDA;
+    ctx->launches += 2;
+    if (ctx->cfg.state_sync == QSR_STATE_RESET) ctx->t_state_origin = t_next;
+    return QSR_OK;
+}
+
 int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
             int64_t *round_start, int64_t *round_len, int64_t cap, int64_t *n_rounds)
 {

@@ -56,6 +56,8 @@ int launch_sync_partial(const SyncParams &p, const LaunchShape &shape, void *str
 int launch_sync_finish(const SyncParams &p, const LaunchShape &shape, void *stream);   // sums -> rows (+ zero)
 int launch_broadcast(float *theta, const float *theta0, int64_t P, int64_t stride, int32_t K,
                      const LaunchShape &shape, void *stream);
+// Both phases through the library's own static scratch; -1 if the sums exceed QSR_STATIC_SCRATCH_FLOATS.
+int launch_sync_static(const SyncParams &p, const LaunchShape &shape, void *stream);
 
 }  // namespace qsr
 #endif

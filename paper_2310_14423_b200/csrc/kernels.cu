@@ -311,3 +311,45 @@ int launch_broadcast(float *theta, const float *theta0, int64_t P, int64_t strid
 }
 
 }  // namespace qsr
+
+// ---------------------------------------------------------------------------------------------- static scratch
+//
+// Scratch of the two-phase synchronization for callers that cannot hand the library a buffer of their own.  It lives
+// in the library image: every GPU that loads the library holds these 4 MiB until the process exits.  In host code the
+// name `g_sync_scratch` is only a handle for the runtime; the address a kernel can use is the one
+// cudaGetSymbolAddress returns for the device that is current at the time.
+static __device__ __align__(256) float g_sync_scratch[QSR_STATIC_SCRATCH_FLOATS];
+
+namespace qsr {
+
+namespace {
+constexpr int kMaxDevices = 64;
+float *g_scratch_addr[kMaxDevices] = {};   // device address of g_sync_scratch, per device ordinal (0 = not yet asked)
+}  // namespace
+
+// The two phases (row sums into the static array, then rows <- sums / K) enqueued back to back on `stream`.
+// Returns 0, a cudaError_t, or -1 when the sums do not fit.  The first call on a device looks the array's device
+// address up; no memory is allocated or freed here.
+int launch_sync_static(const SyncParams &p_in, const LaunchShape &shape, void *stream)
+{
+    if (int64_t(p_in.n_mean) * p_in.P4 > int64_t(QSR_STATIC_SCRATCH_FLOATS)) return -1;
+    int dev = -1;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return int(err);
+    if (dev < 0 || dev >= kMaxDevices) return int(cudaErrorInvalidDevice);
+    float *scratch = g_scratch_addr[dev];
+    if (!scratch) {
+        err = cudaGetSymbolAddress(reinterpret_cast<void **>(&scratch), g_sync_scratch);
+        if (err != cudaSuccess) return int(err);
+        g_scratch_addr[dev] = scratch;
+    }
+    // Every float the second phase reads is written by the first phase of the same call, so nothing left in the
+    // array by an earlier call can leak into this one and nothing has to be cleared.
+    SyncParams p = p_in;
+    p.sum_out = scratch;
+    p.sum_in = scratch;
+    if (int rc = launch_sync_partial(p, shape, stream)) return rc;
+    return launch_sync_finish(p, shape, stream);
+}
+
+}  // namespace qsr
