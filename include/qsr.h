@@ -133,6 +133,13 @@ int qsr_local_step(qsr_ctx *ctx, int64_t t, const float *grads);
  * moves to t_next (the first step of the next round).  One kernel launch; asynchronous. */
 int qsr_sync(qsr_ctx *ctx, int64_t t_next);
 
+/* The last local step of a round and the averaging that ends it (Eq. 1 followed by the All-Reduce line of
+ * Algorithm 2) in ONE launch: the result is bit-identical to qsr_local_step(ctx, t, grads) followed by
+ * qsr_sync(ctx, t_next), but the parameters are read once and written once, so the averaging adds no memory
+ * traffic.  Only state_sync = QSR_STATE_KEEP can be fused; in the other modes this call issues the two launches.
+ * qsr_run uses it for the last step of every round.  Asynchronous. */
+int qsr_local_step_sync(qsr_ctx *ctx, int64_t t, const float *grads, int64_t t_next);
+
 /* The same synchronization split in two for workers sharded over several GPUs: qsr_sync_partial writes
  * sum[i] = sum_k theta[k,i] over this process's rows (and, in AVERAGE mode, the sums of state1 / state2 to
  * sum + P and sum + 2P, each region rounded up to a multiple of 4 floats); the caller all-reduces `sum` over

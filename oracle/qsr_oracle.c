@@ -12,7 +12,9 @@
  *                     2^round(log2 eta_cos(t)) and linear decay (Sec. 4, ablation on schedules).
  *   orc_round_length  Eq. 2: H = max{H_base, floor((alpha/eta_t)^2)} at the round's first global
  *                     step, the warm-up recommendation of Sec. 2 and the forced final
- *                     synchronization H := T - t.
+ *                     synchronization H := T - t; also the general power rule (gamma = 1: H ~ 1/eta,
+ *                     gamma = 3: the cubic rule of App. G), the post-local schedule (Sec. 1) and the
+ *                     modified SWAP schedule (App. H).
  *   orc_local_step    Eq. 1 / the inner loop of Algorithm 2: every worker applies OPT with the
  *                     learning rate of the *global* step; OPT is SGD with heavy-ball momentum and
  *                     L2 weight decay (App. C.1) or AdamW with decoupled weight decay (App. C.2).
@@ -47,8 +49,9 @@
 typedef ORC_REAL real;
 
 enum { ORC_OPT_SGDM = 0, ORC_OPT_ADAMW = 1 };
-enum { ORC_SCHED_COSINE = 0, ORC_SCHED_STEP_POW2 = 1, ORC_SCHED_LINEAR = 2, ORC_SCHED_CONST = 3 };
-enum { ORC_RULE_QSR = 0, ORC_RULE_CONST_H = 1 };
+enum { ORC_SCHED_COSINE = 0, ORC_SCHED_STEP_POW2 = 1, ORC_SCHED_LINEAR = 2, ORC_SCHED_CONST = 3,
+       ORC_SCHED_HALVING = 4, ORC_SCHED_COSINE_HELD = 5 };
+enum { ORC_RULE_QSR = 0, ORC_RULE_CONST_H = 1, ORC_RULE_POWER = 2, ORC_RULE_POST_LOCAL = 3, ORC_RULE_SWAP = 4 };
 enum { ORC_STATE_KEEP = 0, ORC_STATE_AVERAGE = 1, ORC_STATE_RESET = 2 };
 
 typedef struct {
@@ -62,6 +65,10 @@ typedef struct {
     double noise_std;
     int64_t T, T_warmup, H_base;
     uint64_t seed;
+    double gamma;            /* exponent of the power rule H = max{H_base, floor((alpha/eta)^gamma)} (Sec. 2, App. G) */
+    int64_t t_switch;        /* post-local: parallel (H = 1) before it; SWAP variant: one final round after it       */
+    int64_t t_hold, t_period;/* halving schedule: peak until t_hold, then halved every t_period steps (App. G);      */
+                             /* held cosine: the cosine stops decaying at t_hold (App. G)                            */
 } orc_config;
 
 int orc_sizeof_real(void) { return (int)sizeof(real); }
@@ -75,13 +82,22 @@ double orc_lr(const orc_config *c, int64_t t)
     const double pi = 3.14159265358979323846;
     if (t < c->T_warmup)
         return c->eta_max * (double)t / (double)c->T_warmup;
-    double x = (double)(t - c->T_warmup) / (double)(c->T - c->T_warmup);
     if (c->sched == ORC_SCHED_CONST)
         return c->eta_max;
+    if (c->sched == ORC_SCHED_HALVING) {
+        /* App. G: "remains at its peak until [t_hold], after which it is divided by 2 every [t_period]" -- the first
+         * halving happens at t_hold itself (this reading reproduces the 13.2 % and 14.4 % of the step-decay table). */
+        if (t < c->t_hold)
+            return c->eta_max;
+        return ldexp(c->eta_max, -(int)(1 + (t - c->t_hold) / c->t_period));
+    }
+    if (c->sched == ORC_SCHED_COSINE_HELD && t > c->t_hold)
+        t = c->t_hold;       /* the modified cosine of App. G: constant from t_hold on */
+    double x = (double)(t - c->T_warmup) / (double)(c->T - c->T_warmup);
     if (c->sched == ORC_SCHED_LINEAR)
         return c->eta_min + (c->eta_max - c->eta_min) * (1.0 - x);
     double eta_cos = c->eta_min + 0.5 * (c->eta_max - c->eta_min) * (1.0 + cos(pi * x));
-    if (c->sched == ORC_SCHED_COSINE)
+    if (c->sched == ORC_SCHED_COSINE || c->sched == ORC_SCHED_COSINE_HELD)
         return eta_cos;
     /* step schedule: the cosine value rounded to the nearest power of two in the exponent */
     if (eta_cos <= 0.0)
@@ -98,6 +114,16 @@ int64_t orc_round_length(const orc_config *c, int64_t t)
     int64_t H;
     if (c->rule == ORC_RULE_CONST_H) {
         H = c->H_base;
+    } else if (c->rule == ORC_RULE_POST_LOCAL) {
+        /* Post-local schedule (Sec. 1): data-parallel training, i.e. H = 1, until t_switch; then a constant H. */
+        H = t < c->t_switch ? 1 : c->H_base;
+    } else if (c->rule == ORC_RULE_SWAP) {
+        /* The modified SWAP of App. H: constant H_base until t_switch (the last such round is cut there), then
+         * local steps only, with one final averaging at T. */
+        if (t < c->t_switch)
+            H = c->H_base < c->t_switch - t ? c->H_base : c->t_switch - t;
+        else
+            H = c->T - t;
     } else {
         int64_t t_eval = t < c->T_warmup ? c->T_warmup : t;
         double eta = orc_lr(c, t_eval);
@@ -105,7 +131,7 @@ int64_t orc_round_length(const orc_config *c, int64_t t)
             H = c->T - t;
         } else {
             double ratio = c->alpha / eta;
-            double q = ratio * ratio;
+            double q = c->rule == ORC_RULE_POWER ? pow(ratio, c->gamma) : ratio * ratio;
             if (!(q < 4611686018427387904.0)) /* 2^62: beyond any T */
                 H = c->T - t;
             else {

@@ -21,8 +21,8 @@ _LOCK = threading.Lock()
 _LIBS = {}
 
 OPT = {"sgdm": 0, "adamw": 1}
-SCHED = {"cosine": 0, "step_pow2": 1, "linear": 2, "const": 3}
-RULE = {"qsr": 0, "const_h": 1}
+SCHED = {"cosine": 0, "step_pow2": 1, "linear": 2, "const": 3, "halving": 4, "cosine_held": 5}
+RULE = {"qsr": 0, "const_h": 1, "power": 2, "post_local": 3, "swap": 4}
 STATE = {"keep": 0, "average": 1, "reset": 2}
 
 
@@ -31,7 +31,8 @@ class OrcConfig(C.Structure):
                 ("momentum", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double),
                 ("weight_decay", C.c_double), ("eta_max", C.c_double), ("eta_min", C.c_double),
                 ("alpha", C.c_double), ("noise_std", C.c_double),
-                ("T", C.c_int64), ("T_warmup", C.c_int64), ("H_base", C.c_int64), ("seed", C.c_uint64)]
+                ("T", C.c_int64), ("T_warmup", C.c_int64), ("H_base", C.c_int64), ("seed", C.c_uint64),
+                ("gamma", C.c_double), ("t_switch", C.c_int64), ("t_hold", C.c_int64), ("t_period", C.c_int64)]
 
 
 def build(force: bool = False) -> None:
@@ -87,7 +88,9 @@ def config_from(w) -> OrcConfig:
     return OrcConfig(opt=OPT[w.opt], sched=SCHED[w.sched], rule=RULE[w.rule], state_sync=STATE[w.state_sync],
                      momentum=w.momentum, beta1=w.beta1, beta2=w.beta2, eps=w.eps, weight_decay=w.weight_decay,
                      eta_max=w.eta_max, eta_min=w.eta_min, alpha=w.alpha, noise_std=w.noise_std,
-                     T=w.T, T_warmup=w.T_warmup, H_base=w.H_base, seed=w.noise_seed)
+                     T=w.T, T_warmup=w.T_warmup, H_base=w.H_base, seed=w.noise_seed,
+                     gamma=getattr(w, "gamma", 2.0), t_switch=getattr(w, "t_switch", 0),
+                     t_hold=getattr(w, "t_hold", 0), t_period=max(1, getattr(w, "t_period", 1)))
 
 
 def set_threads(n: int) -> None:

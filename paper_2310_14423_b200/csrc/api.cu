@@ -136,6 +136,22 @@ int qsr_local_step(qsr_ctx *ctx, int64_t t, const float *grads)
     return cuda_rc(qsr::launch_step(p, ctx->cfg.opt, ctx->shape, ctx->stream));
 }
 
+int qsr_local_step_sync(qsr_ctx *ctx, int64_t t, const float *grads, int64_t t_next)
+{
+    if (!ctx) return QSR_EINVAL;
+    if (ctx->cfg.state_sync != QSR_STATE_KEEP) {
+        // Averaging or resetting the optimizer state needs the stand-alone kernel: two launches.
+        if (int rc = qsr_local_step(ctx, t, grads)) return rc;
+        return qsr_sync(ctx, t_next);
+    }
+    if (t < 0 || t >= ctx->cfg.T || t < ctx->t_state_origin || t_next < 0 || t_next > ctx->cfg.T) return QSR_ERANGE;
+    if (!grads && !ctx->lambda) return QSR_EINVAL;
+    if (!aligned16(grads)) return QSR_EALIGN;
+    const qsr::StepParams p = step_params(*ctx, t, grads);
+    ctx->launches++;
+    return cuda_rc(qsr::launch_step_mean(p, ctx->cfg.opt, ctx->shape, ctx->stream));
+}
+
 int qsr_sync(qsr_ctx *ctx, int64_t t_next)
 {
     if (!ctx) return QSR_EINVAL;
@@ -206,9 +222,10 @@ int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
     int64_t s = 0;
     for (int64_t t = t_begin; t < t_end;) {
         const int64_t H = qsr::round_length(ctx->cfg, t);       // GetH
-        for (int64_t h = 0; h < H; ++h)
+        for (int64_t h = 0; h + 1 < H; ++h)
             if (int rc = qsr_local_step(ctx, t + h, nullptr)) return rc;
-        if (int rc = qsr_sync(ctx, t + H)) return rc;           // parameter averaging
+        // the round's last step and the parameter averaging, in one launch when the state is kept per worker
+        if (int rc = qsr_local_step_sync(ctx, t + H - 1, nullptr, t + H)) return rc;
         if (s < cap) {
             round_start[s] = t;
             round_len[s] = H;

@@ -44,13 +44,17 @@ struct SyncParams {
 };
 
 struct LaunchShape {
-    int step_threads = 256;
-    int step_rows = 2;
-    int sync_threads = 256;
+    // Defaults from sustained sweeps on B200 at the ViT-B/16 and ResNet-152 shapes (K = 16): 128-thread blocks; rows
+    // in flight per thread 4 for AdamW (three slabs to cover), 2 for SGD.  Grids capped at a few CTAs per SM with a
+    // grid-stride loop were 15-30 % slower than one CTA per 128 columns.
+    int step_threads = 128;
+    int step_rows = 0;        // 0 = pick by optimizer
+    int sync_threads = 128;
 };
 
 // kernels.cu -- each returns a cudaError_t cast to int (0 = success) after enqueueing one kernel.
 int launch_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream);
+int launch_step_mean(const StepParams &p, int opt, const LaunchShape &shape, void *stream);   // step + replica mean
 int launch_sync(const SyncParams &p, const LaunchShape &shape, void *stream);          // mean + write back (+ zero)
 int launch_sync_partial(const SyncParams &p, const LaunchShape &shape, void *stream);  // sums only
 int launch_sync_finish(const SyncParams &p, const LaunchShape &shape, void *stream);   // sums -> rows (+ zero)

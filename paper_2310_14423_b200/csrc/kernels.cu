@@ -94,9 +94,17 @@ __device__ __forceinline__ void opt_update(float &theta, float &a, float &b, flo
 __device__ __forceinline__ float4 ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
 __device__ __forceinline__ void st4(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }
 
+__device__ __forceinline__ float4 add4(float4 x, float4 y) { return make_float4(x.x + y.x, x.y + y.y, x.z + y.z, x.w + y.w); }
+__device__ __forceinline__ float4 div4(float4 x, float d) { return make_float4(x.x / d, x.y / d, x.z / d, x.w / d); }
+
+// One local step of all K workers.  With FUSE_MEAN the step is the last of its round and the kernel also ends the
+// round (Algorithm 2's averaging, state kept per worker): the thread that owns a column sees every worker's new
+// parameters anyway, so it sums them as it goes (k ascending, fp32: the order of the stand-alone sync kernel, hence
+// the same bits) and writes the mean to all K rows instead of the K different values.  The averaging then costs no
+// HBM traffic at all: theta is read once and written once, exactly as in a plain step.
 // No launch bound: the register count decides how many threads fit; a block shape that does not fit is
 // reported by the launch as an error, not silently spilled.
-template <int OPT, bool EXT_GRAD, int ROWS>
+template <int OPT, bool EXT_GRAD, int ROWS, bool FUSE_MEAN>
 __global__ void local_step_kernel(const StepParams p)
 {
     const int64_t n_col = (p.P + 3) >> 2;
@@ -109,6 +117,7 @@ __global__ void local_step_kernel(const StepParams p)
                 lam = ld4(p.lambda + i0);
                 ths = ld4(p.theta_star + i0);
             }
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int k = 0; k < p.K; k += ROWS) {
                 float4 th[ROWS], a[ROWS], b[ROWS], g[ROWS];
 #pragma unroll
@@ -136,28 +145,43 @@ __global__ void local_step_kernel(const StepParams p)
                         opt_update<OPT>(th[r].y, a[r].y, b[r].y, g[r].y, p);
                         opt_update<OPT>(th[r].z, a[r].z, b[r].z, g[r].z, p);
                         opt_update<OPT>(th[r].w, a[r].w, b[r].w, g[r].w, p);
-                        st4(p.theta + e, th[r]);
+                        if (FUSE_MEAN) acc = add4(acc, th[r]);
+                        else st4(p.theta + e, th[r]);
                         st4(p.s1 + e, a[r]);
                         if (OPT == QSR_OPT_ADAMW) st4(p.s2 + e, b[r]);
                     }
                 }
             }
+            if (FUSE_MEAN) {
+                const float4 mean = div4(acc, float(p.K));
+#pragma unroll 4
+                for (int k = 0; k < p.K; ++k) st4(p.theta + int64_t(k) * p.stride + i0, mean);
+            }
         } else {
             // Ragged last column: P is not a multiple of 4.  Scalar accesses, nothing beyond P is touched.
-            const int valid = int(p.P - i0);
-            for (int k = 0; k < p.K; ++k) {
-                float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (!EXT_GRAD) z = noise4(j, p.step, p.worker0 + uint32_t(k), p.key0, p.key1);
-                for (int c = 0; c < valid; ++c) {
-                    const int64_t e = int64_t(k) * p.stride + i0 + c;
+            for (int64_t i = i0; i < p.P; ++i) {
+                const int c = int(i - i0);                                  // 0, 1 or 2
+                float acc = 0.f;
+                for (int k = 0; k < p.K; ++k) {
+                    const int64_t e = int64_t(k) * p.stride + i;
                     float th = p.theta[e], a = p.s1[e], b = OPT == QSR_OPT_ADAMW ? p.s2[e] : 0.f;
-                    const float zc = c == 0 ? z.x : (c == 1 ? z.y : z.z);   // valid <= 3
-                    const float g = EXT_GRAD ? p.grads[e]
-                                             : fmaf(p.sigma, zc, p.lambda[i0 + c] * (th - p.theta_star[i0 + c]));
+                    float g;
+                    if (EXT_GRAD) {
+                        g = p.grads[e];
+                    } else {
+                        const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.key0, p.key1);
+                        const float zc = c == 0 ? z.x : (c == 1 ? z.y : z.z);
+                        g = fmaf(p.sigma, zc, p.lambda[i] * (th - p.theta_star[i]));
+                    }
                     opt_update<OPT>(th, a, b, g, p);
-                    p.theta[e] = th;
+                    if (FUSE_MEAN) acc += th;
+                    else p.theta[e] = th;
                     p.s1[e] = a;
                     if (OPT == QSR_OPT_ADAMW) p.s2[e] = b;
+                }
+                if (FUSE_MEAN) {
+                    const float mean = acc / float(p.K);
+                    for (int k = 0; k < p.K; ++k) p.theta[int64_t(k) * p.stride + i] = mean;
                 }
             }
         }
@@ -165,9 +189,6 @@ __global__ void local_step_kernel(const StepParams p)
 }
 
 // ---------------------------------------------------------------------------------------------- synchronization
-
-__device__ __forceinline__ float4 add4(float4 x, float4 y) { return make_float4(x.x + y.x, x.y + y.y, x.z + y.z, x.w + y.w); }
-__device__ __forceinline__ float4 div4(float4 x, float d) { return make_float4(x.x / d, x.y / d, x.z / d, x.w / d); }
 
 // Sum over rows of one 16-byte column, k ascending, eight loads in flight.
 __device__ __forceinline__ float4 column_sum(const float *slab, int64_t i0, int64_t stride, int K)
@@ -276,28 +297,41 @@ unsigned grid_for(int64_t P, int threads)
     return unsigned(blocks);
 }
 
-template <int OPT, bool EXT>
+template <int OPT, bool EXT, bool FUSE>
 int launch_step_rows(const StepParams &p, const LaunchShape &s, cudaStream_t st)
 {
     const unsigned grid = grid_for(p.P, s.step_threads);
-    switch (s.step_rows) {
-    case 1: local_step_kernel<OPT, EXT, 1><<<grid, s.step_threads, 0, st>>>(p); break;
-    case 2: local_step_kernel<OPT, EXT, 2><<<grid, s.step_threads, 0, st>>>(p); break;
-    case 4: local_step_kernel<OPT, EXT, 4><<<grid, s.step_threads, 0, st>>>(p); break;
-    default: local_step_kernel<OPT, EXT, 8><<<grid, s.step_threads, 0, st>>>(p); break;
+    const int rows = s.step_rows ? s.step_rows : (OPT == QSR_OPT_ADAMW ? 4 : 2);
+    switch (rows) {
+    case 1: local_step_kernel<OPT, EXT, 1, FUSE><<<grid, s.step_threads, 0, st>>>(p); break;
+    case 2: local_step_kernel<OPT, EXT, 2, FUSE><<<grid, s.step_threads, 0, st>>>(p); break;
+    case 4: local_step_kernel<OPT, EXT, 4, FUSE><<<grid, s.step_threads, 0, st>>>(p); break;
+    default: local_step_kernel<OPT, EXT, 8, FUSE><<<grid, s.step_threads, 0, st>>>(p); break;
     }
     return int(cudaGetLastError());
+}
+
+template <bool FUSE>
+int launch_step_any(const StepParams &p, int opt, const LaunchShape &shape, cudaStream_t st)
+{
+    const bool ext = p.grads != nullptr;
+    if (opt == QSR_OPT_SGDM)
+        return ext ? launch_step_rows<QSR_OPT_SGDM, true, FUSE>(p, shape, st)
+                   : launch_step_rows<QSR_OPT_SGDM, false, FUSE>(p, shape, st);
+    return ext ? launch_step_rows<QSR_OPT_ADAMW, true, FUSE>(p, shape, st)
+               : launch_step_rows<QSR_OPT_ADAMW, false, FUSE>(p, shape, st);
 }
 
 }  // namespace
 
 int launch_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream)
 {
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool ext = p.grads != nullptr;
-    if (opt == QSR_OPT_SGDM)
-        return ext ? launch_step_rows<QSR_OPT_SGDM, true>(p, shape, st) : launch_step_rows<QSR_OPT_SGDM, false>(p, shape, st);
-    return ext ? launch_step_rows<QSR_OPT_ADAMW, true>(p, shape, st) : launch_step_rows<QSR_OPT_ADAMW, false>(p, shape, st);
+    return launch_step_any<false>(p, opt, shape, static_cast<cudaStream_t>(stream));
+}
+
+int launch_step_mean(const StepParams &p, int opt, const LaunchShape &shape, void *stream)
+{
+    return launch_step_any<true>(p, opt, shape, static_cast<cudaStream_t>(stream));
 }
 
 int launch_sync(const SyncParams &p, const LaunchShape &shape, void *stream)

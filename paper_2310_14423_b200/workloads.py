@@ -27,8 +27,13 @@ SCHED_COSINE = "cosine"
 SCHED_STEP_POW2 = "step_pow2"
 SCHED_LINEAR = "linear"
 SCHED_CONST = "const"
+SCHED_HALVING = "halving"          # peak until t_hold, then halved every t_period steps (App. G)
+SCHED_COSINE_HELD = "cosine_held"  # cosine that stops decaying at t_hold (App. G)
 RULE_QSR = "qsr"
 RULE_CONST_H = "const_h"
+RULE_POWER = "power"               # H = max(H_base, floor((alpha/eta)^gamma))
+RULE_POST_LOCAL = "post_local"     # H = 1 until t_switch, then H_base
+RULE_SWAP = "swap"                 # H_base until t_switch, then a single round to T
 STATE_KEEP = "keep"
 STATE_AVERAGE = "average"
 STATE_RESET = "reset"
@@ -158,6 +163,10 @@ class Workload:
     data_seed: int = 1          # seed of lambda / theta*
     noise_seed: int = NOISE_SEED_BASE
     worker_offset: int = 0      # global index of this process's first replica (multi-GPU sharding)
+    gamma: float = 2.0          # exponent of the power rule
+    t_switch: int = 0           # switching step of the post-local and SWAP schedules
+    t_hold: int = 0             # halving / held-cosine schedules: last step at the regular value
+    t_period: int = 1           # halving schedule: steps between halvings
 
     @property
     def P(self) -> int:

@@ -87,7 +87,7 @@ def test_tiny_ragged_runs(opt, P):
     orc = G.oracle_on(w, lam, ths)
     ost, oH = orc.run()
     assert np.array_equal(st, ost) and np.array_equal(H, oH)
-    assert launches == w.T + len(st)
+    assert launches == w.T          # the last step of each round carries the averaging
     theta = S.theta[:, :P].cpu().numpy()
     assert (theta == theta[0]).all()
     assert G.rel_err(theta[0], orc.theta[0]) <= G.REL_TOL
@@ -114,7 +114,7 @@ def test_config1_full():
     ost, oH = orc.run()
     assert np.array_equal(st, ost) and np.array_equal(H, oH)
     assert np.array_equal(st + H, ost + oH)            # sync step indices
-    assert len(st) == 203 and launches == 2000 + 203
+    assert len(st) == 203 and launches == 2000
     theta = S.theta.cpu().numpy()
     assert (theta == theta[0]).all()
     assert G.rel_err(theta[0], orc.theta[0]) <= G.REL_TOL
@@ -263,6 +263,34 @@ def test_train_host_equals_context_path():
         with pytest.raises(B.QsrError) as e:
             B.qsr_train_host(cfg, np.zeros(w.P, np.float32), lam, ths, out, small)
         assert e.value.status == B.QSR_ERANGE
+
+
+@pytest.mark.parametrize("opt", [W.OPT_SGDM, W.OPT_ADAMW])
+@pytest.mark.parametrize("K,P", [(3, 1001), (5, 4098), (16, 2051), (1, 7)])
+def test_fused_last_step_equals_step_then_sync_bitwise(opt, K, P):
+    """qsr_local_step_sync (one launch) against qsr_local_step + qsr_sync (two): same bits in every slab."""
+    w = W.tiny_workload(opt, K=K, P=P, T=36)
+    lam, ths, lam_d, ths_d = G.device_inputs(w)
+    A, Bs = G.Slabs(w), G.Slabs(w)
+    ca, cb = G.make_context(w, A, lam_d, ths_d), G.make_context(w, Bs, lam_d, ths_d)
+    t = 0
+    while t < w.T:
+        H = ca.qsr_round_length(t)
+        for h in range(H - 1):
+            ca.qsr_local_step(t + h)
+            cb.qsr_local_step(t + h)
+        ca.qsr_local_step(t + H - 1)
+        ca.qsr_sync(t + H)
+        cb.qsr_local_step_sync(t + H - 1, t + H)
+        t += H
+    torch.cuda.synchronize()
+    assert cb.qsr_launch_count() == w.T and ca.qsr_launch_count() > w.T
+    assert torch.equal(A.theta, Bs.theta) and torch.equal(A.s1, Bs.s1)
+    if opt == W.OPT_ADAMW:
+        assert torch.equal(A.s2, Bs.s2)
+    assert Bs.guards_intact()
+    ca.close()
+    cb.close()
 
 
 def test_nonzero_start_and_set_params():
