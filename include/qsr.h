@@ -40,8 +40,9 @@ typedef enum {
 } qsr_status;
 
 enum { QSR_OPT_SGDM = 0, QSR_OPT_ADAMW = 1 };
-enum { QSR_SCHED_COSINE = 0, QSR_SCHED_STEP_POW2 = 1, QSR_SCHED_LINEAR = 2, QSR_SCHED_CONST = 3 };
-enum { QSR_RULE_QSR = 0, QSR_RULE_CONST_H = 1 };
+enum { QSR_SCHED_COSINE = 0, QSR_SCHED_STEP_POW2 = 1, QSR_SCHED_LINEAR = 2, QSR_SCHED_CONST = 3,
+       QSR_SCHED_HALVING = 4, QSR_SCHED_COSINE_HELD = 5 };
+enum { QSR_RULE_QSR = 0, QSR_RULE_CONST_H = 1, QSR_RULE_POWER = 2, QSR_RULE_POST_LOCAL = 3, QSR_RULE_SWAP = 4 };
 enum { QSR_STATE_KEEP = 0, QSR_STATE_AVERAGE = 1, QSR_STATE_RESET = 2 };
 
 /*
@@ -54,10 +55,15 @@ enum { QSR_STATE_KEEP = 0, QSR_STATE_AVERAGE = 1, QSR_STATE_RESET = 2 };
  *                  n = t + 1 - t_state_origin counts the steps the state has seen.
  * Learning rate eta_t, t in {0..T-1} (Sec. 2): eta_max*t/T_warmup during warm-up, then, with
  *   x = (t - T_warmup)/(T - T_warmup):  COSINE eta_min + (eta_max-eta_min)*(1+cos(pi*x))/2;  STEP_POW2 that value
- *   rounded to 2^round(log2(.)) (Sec. 4, step-decay ablation);  LINEAR eta_min + (eta_max-eta_min)*(1-x);  CONST eta_max.
+ *   rounded to 2^round(log2(.)) (Sec. 4, step-decay ablation);  LINEAR eta_min + (eta_max-eta_min)*(1-x);  CONST eta_max;
+ *   HALVING (App. G) eta_max until t_hold, then eta_max / 2^(1 + (t - t_hold)/t_period) (integer division);
+ *   COSINE_HELD (App. G) the cosine value of min(t, t_hold).
  * Round length (Eq. 2): QSR_RULE_QSR H = max(H_base, floor((alpha/eta_t)^2)) with eta_t taken at the round's first
- *   step, or at t = T_warmup for rounds that start during warm-up (Sec. 2); QSR_RULE_CONST_H H = H_base.  In both
- *   cases H is cut to T - t so that the last round ends at T.
+ *   step, or at t = T_warmup for rounds that start during warm-up (Sec. 2); QSR_RULE_POWER the same with exponent
+ *   gamma, pow(alpha/eta_t, gamma) (Sec. 2; gamma = 1 is H ~ 1/eta, gamma = 3 the cubic rule of App. G);
+ *   QSR_RULE_CONST_H H = H_base; QSR_RULE_POST_LOCAL H = 1 while t < t_switch, then H_base (Sec. 1);
+ *   QSR_RULE_SWAP H = min(H_base, t_switch - t) while t < t_switch, then one round to T (App. H).  In all cases H is
+ *   cut to T - t so that the last round ends at T.
  * Synthetic gradient (stands in for Sample() and back-propagation of Algorithm 2 when no gradient slab is
  *   passed): g[k,i] = lambda[i]*(theta[k,i] - theta_star[i]) + noise_std*z(seed, worker_offset + k, t, i), where z is
  *   a standard normal obtained by Box-Muller from Philox-4x32-10 with counter (i/4 low, i/4 high, t, worker) and
@@ -81,6 +87,10 @@ typedef struct qsr_config {
     int64_t T, T_warmup, H_base;
     int64_t t_state_origin; /* global step at which state1/state2 were last all-zero (0 for a fresh run)    */
     uint64_t seed;
+    double gamma;           /* QSR_RULE_POWER: exponent                                                     */
+    int64_t t_switch;       /* QSR_RULE_POST_LOCAL / QSR_RULE_SWAP: switching step                          */
+    int64_t t_hold;         /* QSR_SCHED_HALVING / QSR_SCHED_COSINE_HELD: see above                         */
+    int64_t t_period;       /* QSR_SCHED_HALVING: steps between halvings (>= 1)                             */
 } qsr_config;
 
 /* ---- host-only schedule (no device, no context) ------------------------------------------------------- */

@@ -18,8 +18,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libqsr.so")
 
 OPT = {"sgdm": 0, "adamw": 1}
-SCHED = {"cosine": 0, "step_pow2": 1, "linear": 2, "const": 3}
-RULE = {"qsr": 0, "const_h": 1}
+SCHED = {"cosine": 0, "step_pow2": 1, "linear": 2, "const": 3, "halving": 4, "cosine_held": 5}
+RULE = {"qsr": 0, "const_h": 1, "power": 2, "post_local": 3, "swap": 4}
 STATE = {"keep": 0, "average": 1, "reset": 2}
 
 QSR_OK, QSR_EINVAL, QSR_EALIGN, QSR_ECUDA, QSR_ERANGE, QSR_ESTATE = 0, -1, -2, -3, -4, -5
@@ -39,7 +39,8 @@ class QsrConfig(C.Structure):
                 ("weight_decay", C.c_double), ("eta_max", C.c_double), ("eta_min", C.c_double),
                 ("alpha", C.c_double), ("noise_std", C.c_double),
                 ("T", C.c_int64), ("T_warmup", C.c_int64), ("H_base", C.c_int64), ("t_state_origin", C.c_int64),
-                ("seed", C.c_uint64)]
+                ("seed", C.c_uint64), ("gamma", C.c_double), ("t_switch", C.c_int64), ("t_hold", C.c_int64),
+                ("t_period", C.c_int64)]
 
 
 class QsrError(RuntimeError):
@@ -110,7 +111,9 @@ def make_config(w, K: Optional[int] = None, row_stride: Optional[int] = None, wo
                      momentum=w.momentum, beta1=w.beta1, beta2=w.beta2, eps=w.eps, weight_decay=w.weight_decay,
                      eta_max=w.eta_max, eta_min=w.eta_min, alpha=w.alpha, noise_std=w.noise_std,
                      T=int(w.T), T_warmup=int(w.T_warmup), H_base=int(w.H_base), t_state_origin=int(t_state_origin),
-                     seed=int(w.noise_seed))
+                     seed=int(w.noise_seed), gamma=float(getattr(w, "gamma", 2.0)),
+                     t_switch=int(getattr(w, "t_switch", 0)), t_hold=int(getattr(w, "t_hold", 0)),
+                     t_period=max(1, int(getattr(w, "t_period", 1))))
 
 
 # ---- host-only schedule ---------------------------------------------------------------------------------

@@ -22,8 +22,12 @@ int check_config(const qsr_config &c)
 {
     if (c.K < 1 || c.P < 1) return QSR_EINVAL;
     if (c.opt != QSR_OPT_SGDM && c.opt != QSR_OPT_ADAMW) return QSR_EINVAL;
-    if (c.sched < QSR_SCHED_COSINE || c.sched > QSR_SCHED_CONST) return QSR_EINVAL;
-    if (c.rule != QSR_RULE_QSR && c.rule != QSR_RULE_CONST_H) return QSR_EINVAL;
+    if (c.sched < QSR_SCHED_COSINE || c.sched > QSR_SCHED_COSINE_HELD) return QSR_EINVAL;
+    if (c.rule < QSR_RULE_QSR || c.rule > QSR_RULE_SWAP) return QSR_EINVAL;
+    if (c.rule == QSR_RULE_POWER && !(std::isfinite(c.gamma) && c.gamma > 0.0)) return QSR_EINVAL;
+    if ((c.rule == QSR_RULE_POST_LOCAL || c.rule == QSR_RULE_SWAP) && (c.t_switch < 0 || c.t_switch > c.T)) return QSR_ERANGE;
+    if (c.sched == QSR_SCHED_HALVING && (c.t_period < 1 || c.t_hold < 0)) return QSR_ERANGE;
+    if (c.sched == QSR_SCHED_COSINE_HELD && c.t_hold < c.T_warmup) return QSR_ERANGE;
     if (c.state_sync < QSR_STATE_KEEP || c.state_sync > QSR_STATE_RESET) return QSR_EINVAL;
     if (!finite_all({c.momentum, c.beta1, c.beta2, c.eps, c.weight_decay, c.eta_max, c.eta_min, c.alpha, c.noise_std}))
         return QSR_EINVAL;
@@ -42,18 +46,26 @@ int check_config(const qsr_config &c)
 double learning_rate(const qsr_config &c, int64_t t)
 {
     if (t < c.T_warmup) return c.eta_max * double(t) / double(c.T_warmup);
-    const double x = double(t - c.T_warmup) / double(c.T - c.T_warmup);
     switch (c.sched) {
     case QSR_SCHED_CONST:
         return c.eta_max;
-    case QSR_SCHED_LINEAR:
-        return c.eta_min + (c.eta_max - c.eta_min) * (1.0 - x);
+    case QSR_SCHED_HALVING: {
+        // Peak until t_hold; the first halving takes effect at t_hold itself, the next ones every t_period steps.
+        if (t < c.t_hold) return c.eta_max;
+        const int64_t halvings = 1 + (t - c.t_hold) / c.t_period;
+        return std::ldexp(c.eta_max, -int(halvings < 2000 ? halvings : 2000));
+    }
+    case QSR_SCHED_COSINE_HELD:
+        if (t > c.t_hold) t = c.t_hold;   // the cosine stops decaying here
+        break;
     default:
         break;
     }
+    const double x = double(t - c.T_warmup) / double(c.T - c.T_warmup);
+    if (c.sched == QSR_SCHED_LINEAR) return c.eta_min + (c.eta_max - c.eta_min) * (1.0 - x);
     const double pi = 3.14159265358979323846;
     const double cosine = c.eta_min + 0.5 * (c.eta_max - c.eta_min) * (1.0 + std::cos(pi * x));
-    if (c.sched == QSR_SCHED_COSINE) return cosine;
+    if (c.sched != QSR_SCHED_STEP_POW2) return cosine;
     // Step schedule: the cosine value with its base-2 logarithm rounded to the nearest integer.
     return cosine > 0.0 ? std::exp2(std::floor(std::log2(cosine) + 0.5)) : 0.0;
 }
@@ -64,11 +76,20 @@ int64_t round_length(const qsr_config &c, int64_t t)
 {
     const int64_t left = c.T - t;
     int64_t H = c.H_base;
-    if (c.rule == QSR_RULE_QSR) {
+    switch (c.rule) {
+    case QSR_RULE_POST_LOCAL:
+        if (t < c.t_switch) H = 1;          // data-parallel phase: a synchronization after every step
+        break;
+    case QSR_RULE_SWAP:
+        if (t >= c.t_switch) H = left;      // local steps only, one final averaging
+        else if (c.t_switch - t < H) H = c.t_switch - t;
+        break;
+    case QSR_RULE_QSR:
+    case QSR_RULE_POWER: {
         const double eta = learning_rate(c, t < c.T_warmup ? c.T_warmup : t);
         if (eta > 0.0) {
             const double ratio = c.alpha / eta;
-            const double q = ratio * ratio;
+            const double q = c.rule == QSR_RULE_POWER ? std::pow(ratio, c.gamma) : ratio * ratio;
             if (q < 4611686018427387904.0) {  // 2^62
                 const int64_t fl = int64_t(std::floor(q));
                 if (fl > H) H = fl;
@@ -78,6 +99,10 @@ int64_t round_length(const qsr_config &c, int64_t t)
         } else {
             H = left;  // the learning rate has reached zero: one round to the end
         }
+        break;
+    }
+    default:
+        break;
     }
     return H < left ? H : left;
 }

@@ -39,8 +39,8 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_config_struct_matches_header_size():
-    # 4 int32 + 2 int64 interleaved as in the header, 9 doubles, 4 int64, 1 uint64: 8 + 16 + 16 + 72 + 32 + 8
-    assert C.sizeof(B.QsrConfig) == 152
+    # 2 int32, 2 int64, 4 int32, 9 doubles, 4 int64, 1 uint64, 1 double, 3 int64: 8 + 16 + 16 + 72 + 32 + 8 + 8 + 24
+    assert C.sizeof(B.QsrConfig) == 184
 
 
 def test_strerror_and_status_codes():
@@ -64,7 +64,11 @@ def test_config_validation():
     assert bad(P=0) == B.QSR_EINVAL
     assert bad(opt=7) == B.QSR_EINVAL
     assert bad(sched=-1) == B.QSR_EINVAL
-    assert bad(rule=2) == B.QSR_EINVAL
+    assert bad(sched=6) == B.QSR_EINVAL
+    assert bad(rule=5) == B.QSR_EINVAL
+    assert bad(rule=2, gamma=0.0) == B.QSR_EINVAL
+    assert bad(rule=3, t_switch=-1) == B.QSR_ERANGE
+    assert bad(sched=4, t_period=0) == B.QSR_ERANGE
     assert bad(state_sync=3) == B.QSR_EINVAL
     assert bad(eta_max=float("nan")) == B.QSR_EINVAL
     assert bad(alpha=float("inf")) == B.QSR_EINVAL
@@ -168,3 +172,33 @@ def test_round_length_pointwise_and_truncation():
         assert B.qsr_config_round_length(cfg, t) == O.round_length(w, t)
     assert B.qsr_config_round_length(cfg, 1999) == 1
     assert B.qsr_config_round_length(cfg, 0) == 4          # (0.2/0.1)^2 is exactly 4 in binary64
+
+
+def test_other_rules_and_schedules_equal_oracle():
+    """Power rule (gamma = 1, 3, 1.5), post-local, modified SWAP; halving and held-cosine schedules (App. G, App. H)."""
+    per_epoch = IMAGENET_TRAIN // 4096
+    vit = W.Workload("vit", 1, W.flat_layout(4), W.OPT_ADAMW, T=300 * per_epoch, T_warmup=10000, eta_max=0.008,
+                     alpha=0.0175, H_base=4)
+    halving = dict(sched=W.SCHED_HALVING, t_hold=150 * per_epoch, t_period=30 * per_epoch)
+    cases = [
+        vit.replace(**halving),
+        vit.replace(rule=W.RULE_POWER, gamma=3.0, alpha=0.0075, **halving),
+        vit.replace(rule=W.RULE_POWER, gamma=3.0, alpha=0.0075, eta_min=1e-6),
+        vit.replace(rule=W.RULE_POWER, gamma=1.0, alpha=0.03),
+        vit.replace(rule=W.RULE_POWER, gamma=1.5, alpha=0.02, H_base=2),
+        vit.replace(sched=W.SCHED_COSINE_HELD, t_hold=250 * per_epoch),
+        vit.replace(sched=W.SCHED_COSINE_HELD, t_hold=250 * per_epoch, rule=W.RULE_POWER, gamma=3.0, alpha=0.0075),
+        vit.replace(rule=W.RULE_POST_LOCAL, t_switch=100 * per_epoch, H_base=8),
+        vit.replace(rule=W.RULE_SWAP, t_switch=280 * per_epoch + 1, H_base=4),
+        W.workload("c1").replace(rule=W.RULE_POWER, gamma=3.0, alpha=0.13),
+    ]
+    for w in cases:
+        st, H = _same_schedule(w)
+        assert H.sum() == w.T
+        cfg = B.make_config(w)
+        for t in range(0, w.T, 4999):
+            assert B.qsr_config_learning_rate(cfg, t) == O.lr(w, t)
+    st, H = _same_schedule(cases[0])
+    assert abs(100.0 * len(st) / cases[0].T - 13.2) <= 0.055      # step-decay table of App. G
+    st, H = _same_schedule(cases[1])
+    assert abs(100.0 * len(st) / cases[1].T - 14.4) <= 0.055
