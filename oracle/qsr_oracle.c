@@ -240,6 +240,36 @@ void orc_local_step(const orc_config *c, int64_t rows, int64_t k0, int64_t n, co
     }
 }
 
+/* ------------------------------------------------------------------ Algorithm 1 (Parallel OPT) */
+
+/* One iteration of the data-parallel baseline: all K workers evaluate their gradient at the SAME parameters
+ * theta [n], the gradients are averaged (the All-Reduce line of Algorithm 1) and ONE optimizer step is taken with
+ * the mean.  grads == NULL: worker k's gradient is lambda*(theta - theta_star) + noise_std * z(seed, k, t, i);
+ * otherwise grads is [K, n].  Returns 0, or -1 if memory for the mean gradient cannot be had. */
+int orc_parallel_step(const orc_config *c, int64_t K, int64_t n, const int64_t *idx,
+                      const real *lambda, const real *theta_star,
+                      real *theta, real *s1, real *s2, const real *grads,
+                      int64_t t, int64_t n_state)
+{
+    real *g_mean = (real *)malloc((size_t)(n > 0 ? n : 1) * sizeof(real));
+    if (!g_mean)
+        return -1;
+    for (int64_t col = 0; col < n; ++col) {
+        const int64_t i = idx ? idx[col] : col;
+        real sum = 0;
+        for (int64_t k = 0; k < K; ++k) {
+            if (grads)
+                sum += grads[k * n + col];
+            else
+                sum += lambda[col] * (theta[col] - theta_star[col]) + (real)(c->noise_std * orc_noise(c->seed, k, t, i));
+        }
+        g_mean[col] = sum / (real)K;
+    }
+    orc_local_step(c, 1, 0, n, idx, lambda, theta_star, theta, s1, s2, g_mean, t, n_state);
+    free(g_mean);
+    return 0;
+}
+
 /* ------------------------------------------------------------------ synchronization */
 
 static void mean_rows(int64_t rows, int64_t n, real *x)

@@ -72,6 +72,8 @@ def _lib(mirror: bool = False):
             lib.orc_noise_fill.argtypes = [C.c_uint64, C.c_int64, C.c_int64, C.c_int64, C.c_int64, p]
             lib.orc_local_step.restype = None
             lib.orc_local_step.argtypes = [cfg, C.c_int64, C.c_int64, C.c_int64, p, p, p, p, p, p, p, C.c_int64, C.c_int64]
+            lib.orc_parallel_step.restype = C.c_int
+            lib.orc_parallel_step.argtypes = [cfg, C.c_int64, C.c_int64, p, p, p, p, p, p, p, C.c_int64, C.c_int64]
             lib.orc_sync.restype = None
             lib.orc_sync.argtypes = [cfg, C.c_int64, C.c_int64, p, p, p]
             lib.orc_run.restype = C.c_int64
@@ -164,6 +166,15 @@ class State:
         _lib(self.mirror).orc_local_step(C.byref(self.cfg), self.rows, self.k0, self.n, _ptr(self.idx),
                                          _ptr(self.lam), _ptr(self.theta_star), _ptr(self.theta), _ptr(self.s1),
                                          _ptr(self.s2), _ptr(g), int(t), int(t - self.t_state_origin))
+
+    def parallel_step(self, t: int, K: int, grads: Optional[np.ndarray] = None) -> None:
+        """Algorithm 1 on row 0 (the single model): K workers' gradients at the same point, averaged, one OPT step."""
+        g = None if grads is None else np.ascontiguousarray(grads, self.dtype)
+        assert g is None or g.shape == (K, self.n)
+        rc = _lib(self.mirror).orc_parallel_step(C.byref(self.cfg), int(K), self.n, _ptr(self.idx), _ptr(self.lam),
+                                                 _ptr(self.theta_star), _ptr(self.theta[0]), _ptr(self.s1[0]),
+                                                 _ptr(self.s2[0]), _ptr(g), int(t), int(t - self.t_state_origin))
+        assert rc == 0
 
     def sync(self, t_next: Optional[int] = None) -> None:
         _lib(self.mirror).orc_sync(C.byref(self.cfg), self.rows, self.n, _ptr(self.theta), _ptr(self.s1), _ptr(self.s2))

@@ -319,3 +319,61 @@ def test_coordinate_subset_equals_the_same_columns_of_the_full_run():
         sub = O.State(w, lam[idx], ths[idx], idx=idx)
         sub.run()
         assert np.array_equal(sub.theta, full.theta[:, idx])
+
+
+# ------------------------------------------------------------------ Algorithm 1 (Parallel OPT)
+
+def test_parallel_opt_equals_torch_with_the_mean_gradient():
+    """Algorithm 1: one model, K gradients at the same point, their mean fed to torch.optim."""
+    for opt in (W.OPT_SGDM, W.OPT_ADAMW):
+        K = 5
+        w = W.tiny_workload(opt, K=K, P=14, T=30, weight_decay=0.02)
+        lam, ths = _inputs(w)
+        lam, ths = lam.astype(np.float64), ths.astype(np.float64)
+        S = O.State(w, lam, ths, rows=1)
+        p = torch.zeros(14, dtype=torch.float64, requires_grad=True)
+        if opt == W.OPT_SGDM:
+            topt = torch.optim.SGD([p], lr=1.0, momentum=w.momentum, weight_decay=w.weight_decay)
+        else:
+            topt = torch.optim.AdamW([p], lr=1.0, betas=(w.beta1, w.beta2), eps=w.eps, weight_decay=w.weight_decay)
+        for t in range(w.T):
+            S.parallel_step(t, K)
+            for g in topt.param_groups:
+                g["lr"] = 0.5 * w.eta_max * (1 + math.cos(math.pi * t / w.T))
+            th = p.detach().numpy()
+            p.grad = torch.from_numpy(np.mean([_grad(w, lam, ths, th, k, t) for k in range(K)], axis=0))
+            topt.step()
+        np.testing.assert_allclose(S.theta[0], p.detach().numpy(), rtol=1e-10, atol=1e-13)
+
+
+def test_local_sgd_with_h1_is_parallel_sgd_also_with_momentum():
+    """Sec. 3: Local SGD with H = 1 is parallel SGD.  With per-worker momentum buffers kept across rounds the mean
+    buffer obeys the parallel recursion, so the statement extends to heavy-ball momentum (not to AdamW)."""
+    K = 4
+    w = W.tiny_workload(W.OPT_SGDM, K=K, P=22, T=40, momentum=0.9, weight_decay=0.01, rule=W.RULE_CONST_H, H_base=1)
+    lam, ths = _inputs(w)
+    local = O.State(w, lam, ths)
+    local.run()
+    par = O.State(w, lam, ths, rows=1)
+    for t in range(w.T):
+        par.parallel_step(t, K)
+    np.testing.assert_allclose(local.theta[0], par.theta[0], rtol=1e-11, atol=1e-13)
+    wa = w.replace(opt=W.OPT_ADAMW, eta_max=0.02)
+    la, pa = O.State(wa, lam, ths), O.State(wa, lam, ths, rows=1)
+    la.run()
+    for t in range(wa.T):
+        pa.parallel_step(t, K)
+    assert np.abs(la.theta[0] - pa.theta[0]).max() > 1e-6
+
+
+def test_parallel_opt_external_gradients():
+    K = 3
+    w = W.tiny_workload(W.OPT_ADAMW, K=K, P=9, T=8)
+    lam, ths = _inputs(w)
+    lam, ths = lam.astype(np.float64), ths.astype(np.float64)
+    A, Bq = O.State(w, lam, ths, rows=1), O.State(w, lam, ths, rows=1)
+    for t in range(w.T):
+        g = np.stack([_grad(w, lam, ths, Bq.theta[0], k, t) for k in range(K)])
+        A.parallel_step(t, K)
+        Bq.parallel_step(t, K, grads=g)
+    np.testing.assert_allclose(A.theta, Bq.theta, rtol=1e-13, atol=1e-15)
