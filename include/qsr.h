@@ -150,6 +150,13 @@ int qsr_sync(qsr_ctx *ctx, int64_t t_next);
  * qsr_run uses it for the last step of every round.  Asynchronous. */
 int qsr_local_step_sync(qsr_ctx *ctx, int64_t t, const float *grads, int64_t t_next);
 
+/* One iteration of Algorithm 1 (Parallel OPT), the data-parallel baseline that synchronizes at every step: the single
+ * model is ROW 0 of params / state1 / state2 (rows 1..K-1 are neither read nor written); the K workers' gradients
+ * are taken at that one point, summed in fp32 for k = 0..K-1, divided by K (the All-Reduce line), and one
+ * optimizer step with learning rate eta_t follows.  grads as in qsr_local_step (NULL: generated; else [K, row_stride]).
+ * With SGD (momentum included, state kept) this is what Local SGD does with H = 1 (Sec. 3).  One launch; asynchronous. */
+int qsr_parallel_step(qsr_ctx *ctx, int64_t t, const float *grads);
+
 /* The same synchronization split in two for workers sharded over several GPUs: qsr_sync_partial writes
  * sum[i] = sum_k theta[k,i] over this process's rows (and, in AVERAGE mode, the sums of state1 / state2 to
  * sum + P and sum + 2P, each region rounded up to a multiple of 4 floats); the caller all-reduces `sum` over

@@ -27,7 +27,7 @@ QSR_STATIC_SCRATCH_FLOATS = 1 << 20
 
 EXPORTS = ("qsr_config_check", "qsr_config_learning_rate", "qsr_config_round_length", "qsr_config_schedule",
            "qsr_workspace_bytes", "qsr_init", "qsr_destroy", "qsr_round_length", "qsr_set_params", "qsr_local_step",
-           "qsr_local_step_sync", "qsr_sync", "qsr_sync_sum_floats", "qsr_sync_partial", "qsr_sync_finish", "qsr_sync_static", "qsr_run", "qsr_launch_count",
+           "qsr_local_step_sync", "qsr_parallel_step", "qsr_sync", "qsr_sync_sum_floats", "qsr_sync_partial", "qsr_sync_finish", "qsr_sync_static", "qsr_run", "qsr_launch_count",
            "qsr_set_launch_shape", "qsr_train_host", "qsr_strerror")
 
 
@@ -73,6 +73,7 @@ def lib():
             "qsr_set_params": (C.c_int, [vp, vp]),
             "qsr_local_step": (C.c_int, [vp, i64, vp]),
             "qsr_local_step_sync": (C.c_int, [vp, i64, vp, i64]),
+            "qsr_parallel_step": (C.c_int, [vp, i64, vp]),
             "qsr_sync": (C.c_int, [vp, i64]),
             "qsr_sync_sum_floats": (i64, [vp]),
             "qsr_sync_partial": (C.c_int, [vp, vp]),
@@ -195,6 +196,9 @@ class Context:
 
     def qsr_local_step_sync(self, t: int, t_next: int, grads=None) -> None:
         _check(lib().qsr_local_step_sync(self._h, int(t), _dptr(grads), int(t_next)), "qsr_local_step_sync")
+
+    def qsr_parallel_step(self, t: int, grads=None) -> None:
+        _check(lib().qsr_parallel_step(self._h, int(t), _dptr(grads)), "qsr_parallel_step")
 
     def qsr_sync(self, t_next: int) -> None:
         _check(lib().qsr_sync(self._h, int(t_next)), "qsr_sync")

@@ -136,6 +136,17 @@ int qsr_local_step(qsr_ctx *ctx, int64_t t, const float *grads)
     return cuda_rc(qsr::launch_step(p, ctx->cfg.opt, ctx->shape, ctx->stream));
 }
 
+int qsr_parallel_step(qsr_ctx *ctx, int64_t t, const float *grads)
+{
+    if (!ctx) return QSR_EINVAL;
+    if (t < 0 || t >= ctx->cfg.T || t < ctx->t_state_origin) return QSR_ERANGE;
+    if (!grads && !ctx->lambda) return QSR_EINVAL;
+    if (!aligned16(grads)) return QSR_EALIGN;
+    const qsr::StepParams p = step_params(*ctx, t, grads);
+    ctx->launches++;
+    return cuda_rc(qsr::launch_parallel_step(p, ctx->cfg.opt, ctx->shape, ctx->stream));
+}
+
 int qsr_local_step_sync(qsr_ctx *ctx, int64_t t, const float *grads, int64_t t_next)
 {
     if (!ctx) return QSR_EINVAL;

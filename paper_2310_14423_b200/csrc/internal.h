@@ -55,6 +55,7 @@ struct LaunchShape {
 // kernels.cu -- each returns a cudaError_t cast to int (0 = success) after enqueueing one kernel.
 int launch_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream);
 int launch_step_mean(const StepParams &p, int opt, const LaunchShape &shape, void *stream);   // step + replica mean
+int launch_parallel_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream);  // Algorithm 1, row 0
 int launch_sync(const SyncParams &p, const LaunchShape &shape, void *stream);          // mean + write back (+ zero)
 int launch_sync_partial(const SyncParams &p, const LaunchShape &shape, void *stream);  // sums only
 int launch_sync_finish(const SyncParams &p, const LaunchShape &shape, void *stream);   // sums -> rows (+ zero)

@@ -188,8 +188,6 @@ __global__ void local_step_kernel(const StepParams p)
     }
 }
 
-// ---------------------------------------------------------------------------------------------- synchronization
-
 // Sum over rows of one 16-byte column, k ascending, eight loads in flight.
 __device__ __forceinline__ float4 column_sum(const float *slab, int64_t i0, int64_t stride, int K)
 {
@@ -205,6 +203,71 @@ __device__ __forceinline__ float4 column_sum(const float *slab, int64_t i0, int6
     for (; k < K; ++k) acc = add4(acc, ld4(slab + int64_t(k) * stride + i0));
     return acc;
 }
+
+// ---------------------------------------------------------------------------------------------- Algorithm 1
+
+// Parallel OPT: the single model lives in row 0 of the slabs; the K workers' gradients are all taken at that one
+// point, summed for k = 0..K-1 and divided by K (the All-Reduce line of Algorithm 1), and one optimizer step follows.
+// HBM traffic is that of one row (plus the K gradient rows when they come from a slab); with generated gradients the
+// kernel is bound by the K noise evaluations per coordinate, not by memory.
+template <int OPT, bool EXT_GRAD>
+__global__ void parallel_step_kernel(const StepParams p)
+{
+    const int64_t n_col = (p.P + 3) >> 2;
+    const int64_t grid_stride = int64_t(gridDim.x) * blockDim.x;
+    const float Kf = float(p.K);
+    for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < n_col; j += grid_stride) {
+        const int64_t i0 = j << 2;
+        if (i0 + 4 <= p.P) {
+            float4 th = ld4(p.theta + i0), a = ld4(p.s1 + i0), b = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (OPT == QSR_OPT_ADAMW) b = ld4(p.s2 + i0);
+            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (EXT_GRAD) {
+                sum = column_sum(p.grads, i0, p.stride, p.K);
+            } else {
+                const float4 lam = ld4(p.lambda + i0), ths = ld4(p.theta_star + i0);
+                const float4 pull = make_float4(lam.x * (th.x - ths.x), lam.y * (th.y - ths.y),
+                                                lam.z * (th.z - ths.z), lam.w * (th.w - ths.w));
+                for (int k = 0; k < p.K; ++k) {
+                    const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.key0, p.key1);
+                    sum.x += fmaf(p.sigma, z.x, pull.x);
+                    sum.y += fmaf(p.sigma, z.y, pull.y);
+                    sum.z += fmaf(p.sigma, z.z, pull.z);
+                    sum.w += fmaf(p.sigma, z.w, pull.w);
+                }
+            }
+            const float4 g = div4(sum, Kf);
+            opt_update<OPT>(th.x, a.x, b.x, g.x, p);
+            opt_update<OPT>(th.y, a.y, b.y, g.y, p);
+            opt_update<OPT>(th.z, a.z, b.z, g.z, p);
+            opt_update<OPT>(th.w, a.w, b.w, g.w, p);
+            st4(p.theta + i0, th);
+            st4(p.s1 + i0, a);
+            if (OPT == QSR_OPT_ADAMW) st4(p.s2 + i0, b);
+        } else {
+            for (int64_t i = i0; i < p.P; ++i) {
+                const int c = int(i - i0);
+                float th = p.theta[i], a = p.s1[i], b = OPT == QSR_OPT_ADAMW ? p.s2[i] : 0.f;
+                float sum = 0.f;
+                for (int k = 0; k < p.K; ++k) {
+                    if (EXT_GRAD) {
+                        sum += p.grads[int64_t(k) * p.stride + i];
+                    } else {
+                        const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.key0, p.key1);
+                        const float zc = c == 0 ? z.x : (c == 1 ? z.y : z.z);
+                        sum += fmaf(p.sigma, zc, p.lambda[i] * (th - p.theta_star[i]));
+                    }
+                }
+                opt_update<OPT>(th, a, b, sum / Kf, p);
+                p.theta[i] = th;
+                p.s1[i] = a;
+                if (OPT == QSR_OPT_ADAMW) p.s2[i] = b;
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------- synchronization
 
 // One array's share of a synchronization for the column (or ragged tail) that starts at coordinate i0.
 // MODE 0: mean of the rows, written back to every row (the whole synchronization on one GPU).
@@ -332,6 +395,21 @@ int launch_step(const StepParams &p, int opt, const LaunchShape &shape, void *st
 int launch_step_mean(const StepParams &p, int opt, const LaunchShape &shape, void *stream)
 {
     return launch_step_any<true>(p, opt, shape, static_cast<cudaStream_t>(stream));
+}
+
+int launch_parallel_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const unsigned grid = grid_for(p.P, shape.step_threads);
+    const bool ext = p.grads != nullptr;
+    if (opt == QSR_OPT_SGDM) {
+        if (ext) parallel_step_kernel<QSR_OPT_SGDM, true><<<grid, shape.step_threads, 0, st>>>(p);
+        else parallel_step_kernel<QSR_OPT_SGDM, false><<<grid, shape.step_threads, 0, st>>>(p);
+    } else {
+        if (ext) parallel_step_kernel<QSR_OPT_ADAMW, true><<<grid, shape.step_threads, 0, st>>>(p);
+        else parallel_step_kernel<QSR_OPT_ADAMW, false><<<grid, shape.step_threads, 0, st>>>(p);
+    }
+    return int(cudaGetLastError());
 }
 
 int launch_sync(const SyncParams &p, const LaunchShape &shape, void *stream)
