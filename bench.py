@@ -38,11 +38,13 @@ UNIT = "param-updates/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic of the dominant kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum per launch),
-# stated per element-update so that it scales to any launch; valid only for the kernel source it was taken from.
+# DRAM traffic of the dominant kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum per launch,
+# taken on the 2^23-parameter variants c4s / c3s and stated per element-update: the kernel streams every element
+# once, so traffic grows in proportion to K*P).  Valid only for the kernel source it was taken from: the hash covers
+# the noise generator, the optimizer update and local_step_kernel in csrc/kernels.cu.
 NCU_TRAFFIC = {
-    "kernels_cu_sha256": None,          # sha256 of csrc/kernels.cu at capture time
-    "local_step_adamw_bytes_per_update": None,
+    "step_source_sha256": "eff7b805a4e9d29a8d1fddd775f0803c9dd528bb49ecc555ef184563b06a504e",
+    "bytes_per_update": {"adamw": 24.077, "sgdm": 16.076},
 }
 
 
@@ -66,9 +68,15 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def kernels_hash():
-    with open(os.path.join(ROOT, "paper_2310_14423_b200", "csrc", "kernels.cu"), "rb") as f:
-        return hashlib.sha256(f.read()).hexdigest()
+def step_source_hash():
+    with open(os.path.join(ROOT, "paper_2310_14423_b200", "csrc", "kernels.cu")) as f:
+        text = f.read()
+    bar = "// " + "-" * 94 + " "
+    try:
+        region = text[text.index(bar + "noise"):text.index("// Sum over rows of one 16-byte column")]
+    except ValueError:
+        return None
+    return hashlib.sha256(region.encode()).hexdigest()
 
 
 class ClockSampler:
@@ -372,9 +380,8 @@ def main():
     step_bytes = step_bytes_per_update(w) * K_local * w.P
     step_gbs = step_bytes / (step_ms * 1e-3) / 1e9
     traffic = None
-    if NCU_TRAFFIC["kernels_cu_sha256"] == kernels_hash() and NCU_TRAFFIC["local_step_adamw_bytes_per_update"] \
-            and w.opt == "adamw":
-        traffic = NCU_TRAFFIC["local_step_adamw_bytes_per_update"] * K_local * w.P
+    if NCU_TRAFFIC["step_source_sha256"] == step_source_hash():
+        traffic = NCU_TRAFFIC["bytes_per_update"][w.opt] * K_local * w.P
     roofline = {"bound": "hbm", "kernel": "local_step_kernel", "achieved": step_gbs, "peak": peak, "unit": "GB/s",
                 "frac": step_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
                 "frac_of_nominal_8TBps": step_gbs / NOMINAL_HBM_GBS,
