@@ -57,6 +57,8 @@ def parse_args():
     ap.add_argument("--workload", default="c4")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sharded-path", action="store_true",
+                    help="on one GPU, still end rounds the multi-GPU way (partial sums, all-reduce of one rank, finish)")
     return ap.parse_args()
 
 
@@ -233,7 +235,8 @@ def main():
     s2 = torch.zeros(K_local, P4, device=dev) if w.opt == W.OPT_ADAMW else None
     stream = torch.cuda.current_stream().cuda_stream
     cfg = B.make_config(w, K=K_local, row_stride=P4)
-    sums = torch.zeros(3 * P4, device=dev) if world > 1 else None
+    sharded_path = world > 1 or args.sharded_path      # rounds end with partial sums + all-reduce + finish
+    sums = torch.zeros(3 * P4, device=dev) if sharded_path else None
 
     def all_reduce(buf):
         if world > 1:
@@ -247,7 +250,7 @@ def main():
         return B.Context(cfg, theta, s1, s2, lam, ths, stream=stream)
 
     def do_sync(ctx, t_next):
-        if world == 1:
+        if not sharded_path:
             ctx.qsr_sync(t_next)
         else:
             ctx.qsr_sync_partial(sums)
@@ -277,7 +280,7 @@ def main():
     ev[0].record()
     n_ev = 1
     for t in range(steps):
-        if t + 1 in ends and world == 1:
+        if t + 1 in ends and not sharded_path:
             ctx.qsr_local_step_sync(t, t + 1)     # last step of a round: step and averaging in one launch
             ev[n_ev].record()
             n_ev += 1
@@ -332,7 +335,7 @@ def main():
         out_h = torch.empty(w.P, dtype=torch.float32).pin_memory()
         t_end = min(w.T, steps)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        if world == 1:
+        if not sharded_path:
             # the slabs above are released first: qsr_train_host works in one caller-owned workspace
             theta = s1 = s2 = None
             torch.cuda.empty_cache()
@@ -345,7 +348,8 @@ def main():
             e2e_ms = e0.elapsed_time(e1)
             done = int(r_st[-1] + r_H[-1])      # whole rounds: stops at the first round end at or after t_end
         else:
-            dist.barrier()
+            if world > 1:
+                dist.barrier()
             torch.cuda.synchronize()
             e0.record()
             lam[:w.P].copy_(lam_p, non_blocking=True)
@@ -362,15 +366,17 @@ def main():
             out_h.copy_(theta[0, :w.P], non_blocking=True)
             e1.record()
             torch.cuda.synchronize()
-            dist.barrier()
             ctx.close()
             done = rounds[-1][0] + rounds[-1][1]
-            tmax = torch.tensor([e0.elapsed_time(e1)], device=dev, dtype=torch.float64)
-            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-            e2e_ms = float(tmax.item())
+            e2e_ms = e0.elapsed_time(e1)
+            if world > 1:
+                dist.barrier()
+                tmax = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+                dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+                e2e_ms = float(tmax.item())
         e2e = {"value": K_total * w.P * done / (e2e_ms * 1e-3), "unit": UNIT, "steps": done,
                "h2d_bytes_per_step": 3 * w.P * 4 / done, "d2h_bytes_per_step": w.P * 4 / done,
-               "api": "qsr_train_host" if world == 1 else "sharded.run_rounds"}
+               "api": "sharded.run_rounds" if sharded_path else "qsr_train_host"}
 
     if rank != 0:
         dist.destroy_process_group()
@@ -388,7 +394,7 @@ def main():
                 "algorithmic_bytes_per_launch": step_bytes, "avg_launch_ms": step_ms}
     kernels = {"local_step": {"launches": int((kinds == "step").sum()), "avg_ms": step_ms, "GBps": step_gbs,
                               "frac_of_measured": step_gbs / peak}}
-    if sync_ms is not None and world == 1:
+    if sync_ms is not None and not sharded_path:
         # fused: the round's last step also averages; its traffic is that of a plain step
         fused_gbs = step_bytes / (sync_ms * 1e-3) / 1e9
         kernels["local_step_with_mean"] = {"launches": n_syncs, "avg_ms": sync_ms, "GBps": fused_gbs,
@@ -399,7 +405,7 @@ def main():
         kernels["sync"] = {"launches_outside_window": 20, "avg_ms": sync_alone_ms, "GBps": sa_gbs,
                            "frac_of_measured": sa_gbs / peak, "frac_of_nominal_8TBps": sa_gbs / NOMINAL_HBM_GBS,
                            "note": "stand-alone replica-mean kernel (used when the state is averaged or reset)"}
-    if sync_ms is not None and world > 1:
+    if sync_ms is not None and sharded_path:
         sync_bytes = 8.0 * K_local * w.P + 8.0 * w.P
         sync_gbs = sync_bytes / (sync_ms * 1e-3) / 1e9
         kernels["sync"] = {"launches": n_syncs, "avg_ms": sync_ms, "GBps": sync_gbs, "frac_of_measured": sync_gbs / peak,
@@ -414,7 +420,7 @@ def main():
         "config": {"workload": label, "K_per_gpu": K_local, "K_total": K_total, "P": w.P, "opt": w.opt, "T": w.T,
                    "window": f"global steps [0,{steps}) of the schedule", "syncs_in_window": n_syncs,
                    "l2": "inputs larger than L2 (every launch streams the whole slabs)",
-                   "parallelism": f"replica-sharded dp{world}" if world > 1 else "1 GPU, replicas as slab rows"},
+                   "parallelism": f"replica-sharded dp{world}" if sharded_path else "1 GPU, replicas as slab rows"},
         "roofline": roofline, "kernels": kernels, "gpu_launches": int(launches), "clocks": clocks,
     }
     if e2e is not None:

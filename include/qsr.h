@@ -128,6 +128,15 @@ int qsr_destroy(qsr_ctx *ctx);
 /* Same as qsr_config_round_length on the context's configuration: GetH of Algorithm 2. */
 int64_t qsr_round_length(const qsr_ctx *ctx, int64_t t);
 
+/* Per-tensor weight decay.  The paper uses one weight-decay value for the whole model (App. C); recipes that exempt
+ * normalization and bias tensors are common, so each tensor of the flattened parameter set may carry a factor on it.
+ * tensor_end_dev [n_tensors] (device, int64): one past the last coordinate of each tensor, ascending, every entry a
+ * multiple of 4 except the last, which is P; wd_scale_dev [n_tensors] (device, float): the factor (0 switches weight
+ * decay off for that tensor, 1 leaves it).  Both arrays are borrowed until qsr_destroy or the next call;
+ * n_tensors = 0 restores the uniform weight decay.  The library does not read the arrays on the host, so a table that
+ * breaks these rules is not detected. */
+int qsr_set_tensor_table(qsr_ctx *ctx, int32_t n_tensors, const int64_t *tensor_end_dev, const float *wd_scale_dev);
+
 /* theta[k, :] <- theta0_dev[0..P) for every worker k: "each worker gets a local copy of the global iterate"
  * (Sec. 2).  Asynchronous. */
 int qsr_set_params(qsr_ctx *ctx, const float *theta0_dev);

@@ -69,6 +69,8 @@ typedef struct {
     int64_t t_switch;        /* post-local: parallel (H = 1) before it; SWAP variant: one final round after it       */
     int64_t t_hold, t_period;/* halving schedule: peak until t_hold, then halved every t_period steps (App. G);      */
                              /* held cosine: the cosine stops decaying at t_hold (App. G)                            */
+    const double *wd_scale;  /* NULL, or one factor on the weight decay per column (per-tensor weight decay; the     */
+                             /* paper uses one value for the whole model, App. C)                                    */
 } orc_config;
 
 int orc_sizeof_real(void) { return (int)sizeof(real); }
@@ -208,7 +210,6 @@ void orc_local_step(const orc_config *c, int64_t rows, int64_t k0, int64_t n, co
                     int64_t t, int64_t n_state)
 {
     const real eta = (real)orc_lr(c, t);
-    const real wd = (real)c->weight_decay;
     const real mu = (real)c->momentum;
     const real b1 = (real)c->beta1, b2 = (real)c->beta2, eps = (real)c->eps;
     const real bc1 = (real)(1.0 - pow(c->beta1, (double)(n_state + 1)));
@@ -219,6 +220,7 @@ void orc_local_step(const orc_config *c, int64_t rows, int64_t k0, int64_t n, co
         for (int64_t col = 0; col < n; ++col) {
             const int64_t i = idx ? idx[col] : col;
             const int64_t e = r * n + col;
+            const real wd = (real)(c->weight_decay * (c->wd_scale ? c->wd_scale[col] : 1.0));
             real g;
             if (grads)
                 g = grads[e];

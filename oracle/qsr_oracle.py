@@ -32,7 +32,8 @@ class OrcConfig(C.Structure):
                 ("weight_decay", C.c_double), ("eta_max", C.c_double), ("eta_min", C.c_double),
                 ("alpha", C.c_double), ("noise_std", C.c_double),
                 ("T", C.c_int64), ("T_warmup", C.c_int64), ("H_base", C.c_int64), ("seed", C.c_uint64),
-                ("gamma", C.c_double), ("t_switch", C.c_int64), ("t_hold", C.c_int64), ("t_period", C.c_int64)]
+                ("gamma", C.c_double), ("t_switch", C.c_int64), ("t_hold", C.c_int64), ("t_period", C.c_int64),
+                ("wd_scale", C.c_void_p)]
 
 
 def build(force: bool = False) -> None:
@@ -144,7 +145,8 @@ class State:
     """Parameters and optimizer state of K workers on a set of coordinates, in the oracle's precision."""
 
     def __init__(self, w, lam: np.ndarray, theta_star: np.ndarray, idx: Optional[np.ndarray] = None,
-                 mirror: bool = False, rows: Optional[int] = None, k0: int = 0):
+                 mirror: bool = False, rows: Optional[int] = None, k0: int = 0,
+                 wd_scale: Optional[np.ndarray] = None):
         self.w = w
         self.mirror = mirror
         self.dtype = np.float32 if mirror else np.float64
@@ -160,6 +162,11 @@ class State:
         self.s2 = np.zeros((self.rows, self.n), self.dtype)
         self.t_state_origin = 0
         self.cfg = config_from(w)
+        self.wd_scale = None
+        if wd_scale is not None:                       # one weight-decay factor per column, always binary64
+            self.wd_scale = np.ascontiguousarray(wd_scale, np.float64)
+            assert self.wd_scale.shape == (self.n,)
+            self.cfg.wd_scale = self.wd_scale.ctypes.data
 
     def local_step(self, t: int, grads: Optional[np.ndarray] = None) -> None:
         g = None if grads is None else np.ascontiguousarray(grads, self.dtype)

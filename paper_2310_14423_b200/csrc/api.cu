@@ -17,6 +17,9 @@ struct qsr_ctx {
     int64_t t_state_origin;
     int64_t launches;
     bool partial_pending;
+    int32_t n_tensors;
+    const int64_t *tensor_end;
+    const float *wd_scale;
 };
 
 namespace {
@@ -51,6 +54,7 @@ qsr::StepParams step_params(const qsr_ctx &x, int64_t t, const float *grads)
     p.step_size = float(eta / bc1);
     p.inv_sqrt_bc2 = float(1.0 / std::sqrt(bc2));
     p.eps = float(c.eps);
+    p.n_tensors = x.n_tensors; p.tensor_end = x.tensor_end; p.wd_scale = x.wd_scale;
     return p;
 }
 
@@ -99,6 +103,7 @@ int qsr_init(qsr_ctx **out, const qsr_config *cfg, float *params, float *state1,
     x->t_state_origin = cfg->t_state_origin;
     x->launches = 0;
     x->partial_pending = false;
+    x->n_tensors = 0; x->tensor_end = nullptr; x->wd_scale = nullptr;
     *out = x;
     return QSR_OK;
 }
@@ -134,6 +139,19 @@ int qsr_local_step(qsr_ctx *ctx, int64_t t, const float *grads)
     const qsr::StepParams p = step_params(*ctx, t, grads);
     ctx->launches++;
     return cuda_rc(qsr::launch_step(p, ctx->cfg.opt, ctx->shape, ctx->stream));
+}
+
+int qsr_set_tensor_table(qsr_ctx *ctx, int32_t n_tensors, const int64_t *tensor_end_dev, const float *wd_scale_dev)
+{
+    if (!ctx || n_tensors < 0) return QSR_EINVAL;
+    if (n_tensors == 0) {
+        ctx->n_tensors = 0; ctx->tensor_end = nullptr; ctx->wd_scale = nullptr;
+        return QSR_OK;
+    }
+    if (!tensor_end_dev || !wd_scale_dev) return QSR_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(tensor_end_dev) & 7u) || (reinterpret_cast<uintptr_t>(wd_scale_dev) & 3u)) return QSR_EALIGN;
+    ctx->n_tensors = n_tensors; ctx->tensor_end = tensor_end_dev; ctx->wd_scale = wd_scale_dev;
+    return QSR_OK;
 }
 
 int qsr_parallel_step(qsr_ctx *ctx, int64_t t, const float *grads)

@@ -72,11 +72,13 @@ __device__ __forceinline__ float4 noise4(int64_t j, uint32_t step, uint32_t work
 
 // ---------------------------------------------------------------------------------------------- OPT (Eq. 1)
 
+// `wdv` is the weight-decay scalar of this coordinate's tensor: wd for SGD, eta*wd for AdamW, each times the
+// tensor's scale (1 when no tensor table is set).
 template <int OPT>
-__device__ __forceinline__ void opt_update(float &theta, float &a, float &b, float g, const StepParams &p)
+__device__ __forceinline__ void opt_update(float &theta, float &a, float &b, float g, const StepParams &p, float wdv)
 {
     if (OPT == QSR_OPT_SGDM) {
-        g = fmaf(p.wd, theta, g);          // L2 weight decay enters the gradient
+        g = fmaf(wdv, theta, g);           // L2 weight decay enters the gradient
         a = fmaf(p.mu, a, g);              // heavy-ball buffer
         theta = fmaf(-p.eta, a, theta);
     } else {
@@ -87,8 +89,24 @@ __device__ __forceinline__ void opt_update(float &theta, float &a, float &b, flo
         // keep only ~2^-24 of absolute precision on a term of size eta*wd, and the product theta*(1 - eta*wd) has
         // near-ties that round the same way step after step when theta sits just above a power of two; both show up
         // as a drift of a few 1e-5 over thousands of small steps.  The decay and the update are summed first instead.
-        theta -= fmaf(p.eta_wd, theta, p.step_size * __fdividef(a, denom));
+        theta -= fmaf(wdv, theta, p.step_size * __fdividef(a, denom));
     }
+}
+
+// Weight-decay scalar for the column that starts at coordinate i0: binary search of the tensor that holds it
+// (tensor_end is ascending, every entry but the last a multiple of 4, so a column never straddles two tensors).
+template <int OPT>
+__device__ __forceinline__ float weight_decay_at(const StepParams &p, int64_t i0)
+{
+    const float base = OPT == QSR_OPT_SGDM ? p.wd : p.eta_wd;
+    if (p.n_tensors == 0) return base;
+    int lo = 0, hi = p.n_tensors - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(p.tensor_end + mid) > i0) hi = mid;
+        else lo = mid + 1;
+    }
+    return base * __ldg(p.wd_scale + lo);
 }
 
 __device__ __forceinline__ float4 ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
@@ -111,6 +129,7 @@ __global__ void local_step_kernel(const StepParams p)
     const int64_t grid_stride = int64_t(gridDim.x) * blockDim.x;
     for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < n_col; j += grid_stride) {
         const int64_t i0 = j << 2;
+        const float wdv = weight_decay_at<OPT>(p, i0);
         if (i0 + 4 <= p.P) {
             float4 lam = make_float4(0.f, 0.f, 0.f, 0.f), ths = lam;
             if (!EXT_GRAD) {
@@ -141,10 +160,10 @@ __global__ void local_step_kernel(const StepParams p)
                             g[r].z = fmaf(p.sigma, z.z, lam.z * (th[r].z - ths.z));
                             g[r].w = fmaf(p.sigma, z.w, lam.w * (th[r].w - ths.w));
                         }
-                        opt_update<OPT>(th[r].x, a[r].x, b[r].x, g[r].x, p);
-                        opt_update<OPT>(th[r].y, a[r].y, b[r].y, g[r].y, p);
-                        opt_update<OPT>(th[r].z, a[r].z, b[r].z, g[r].z, p);
-                        opt_update<OPT>(th[r].w, a[r].w, b[r].w, g[r].w, p);
+                        opt_update<OPT>(th[r].x, a[r].x, b[r].x, g[r].x, p, wdv);
+                        opt_update<OPT>(th[r].y, a[r].y, b[r].y, g[r].y, p, wdv);
+                        opt_update<OPT>(th[r].z, a[r].z, b[r].z, g[r].z, p, wdv);
+                        opt_update<OPT>(th[r].w, a[r].w, b[r].w, g[r].w, p, wdv);
                         if (FUSE_MEAN) acc = add4(acc, th[r]);
                         else st4(p.theta + e, th[r]);
                         st4(p.s1 + e, a[r]);
@@ -173,7 +192,7 @@ __global__ void local_step_kernel(const StepParams p)
                         const float zc = c == 0 ? z.x : (c == 1 ? z.y : z.z);
                         g = fmaf(p.sigma, zc, p.lambda[i] * (th - p.theta_star[i]));
                     }
-                    opt_update<OPT>(th, a, b, g, p);
+                    opt_update<OPT>(th, a, b, g, p, wdv);
                     if (FUSE_MEAN) acc += th;
                     else p.theta[e] = th;
                     p.s1[e] = a;
@@ -218,6 +237,7 @@ __global__ void parallel_step_kernel(const StepParams p)
     const float Kf = float(p.K);
     for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < n_col; j += grid_stride) {
         const int64_t i0 = j << 2;
+        const float wdv = weight_decay_at<OPT>(p, i0);
         if (i0 + 4 <= p.P) {
             float4 th = ld4(p.theta + i0), a = ld4(p.s1 + i0), b = make_float4(0.f, 0.f, 0.f, 0.f);
             if (OPT == QSR_OPT_ADAMW) b = ld4(p.s2 + i0);
@@ -237,10 +257,10 @@ __global__ void parallel_step_kernel(const StepParams p)
                 }
             }
             const float4 g = div4(sum, Kf);
-            opt_update<OPT>(th.x, a.x, b.x, g.x, p);
-            opt_update<OPT>(th.y, a.y, b.y, g.y, p);
-            opt_update<OPT>(th.z, a.z, b.z, g.z, p);
-            opt_update<OPT>(th.w, a.w, b.w, g.w, p);
+            opt_update<OPT>(th.x, a.x, b.x, g.x, p, wdv);
+            opt_update<OPT>(th.y, a.y, b.y, g.y, p, wdv);
+            opt_update<OPT>(th.z, a.z, b.z, g.z, p, wdv);
+            opt_update<OPT>(th.w, a.w, b.w, g.w, p, wdv);
             st4(p.theta + i0, th);
             st4(p.s1 + i0, a);
             if (OPT == QSR_OPT_ADAMW) st4(p.s2 + i0, b);
@@ -258,7 +278,7 @@ __global__ void parallel_step_kernel(const StepParams p)
                         sum += fmaf(p.sigma, zc, p.lambda[i] * (th - p.theta_star[i]));
                     }
                 }
-                opt_update<OPT>(th, a, b, sum / Kf, p);
+                opt_update<OPT>(th, a, b, sum / Kf, p, wdv);
                 p.theta[i] = th;
                 p.s1[i] = a;
                 if (OPT == QSR_OPT_ADAMW) p.s2[i] = b;

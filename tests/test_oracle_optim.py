@@ -377,3 +377,31 @@ def test_parallel_opt_external_gradients():
         A.parallel_step(t, K)
         Bq.parallel_step(t, K, grads=g)
     np.testing.assert_allclose(A.theta, Bq.theta, rtol=1e-13, atol=1e-15)
+
+
+def test_per_tensor_weight_decay_equals_torch_param_groups():
+    """Two 'tensors', one with the run's weight decay and one exempt (factor 0), against torch parameter groups."""
+    for opt in (W.OPT_SGDM, W.OPT_ADAMW):
+        w = W.tiny_workload(opt, K=1, P=12, T=25, weight_decay=0.1)
+        lam, ths = _inputs(w)
+        lam, ths = lam.astype(np.float64), ths.astype(np.float64)
+        scale = np.array([1.0] * 8 + [0.0] * 4)
+        S = O.State(w, lam, ths, wd_scale=scale)
+        S.run()
+        pa = torch.zeros(8, dtype=torch.float64, requires_grad=True)
+        pb = torch.zeros(4, dtype=torch.float64, requires_grad=True)
+        groups = [{"params": [pa], "weight_decay": 0.1}, {"params": [pb], "weight_decay": 0.0}]
+        topt = (torch.optim.SGD(groups, lr=1.0, momentum=w.momentum) if opt == W.OPT_SGDM
+                else torch.optim.AdamW(groups, lr=1.0, betas=(w.beta1, w.beta2), eps=w.eps))
+        for t in range(w.T):
+            for g in topt.param_groups:
+                g["lr"] = 0.5 * w.eta_max * (1 + math.cos(math.pi * t / w.T))
+            th = np.concatenate([pa.detach().numpy(), pb.detach().numpy()])
+            g = _grad(w, lam, ths, th, 0, t)
+            pa.grad, pb.grad = torch.from_numpy(g[:8].copy()), torch.from_numpy(g[8:].copy())
+            topt.step()
+        got = np.concatenate([pa.detach().numpy(), pb.detach().numpy()])
+        np.testing.assert_allclose(S.theta[0], got, rtol=1e-10, atol=1e-13)
+        plain = O.State(w, lam, ths)
+        plain.run()
+        assert np.abs(plain.theta[0, 8:] - S.theta[0, 8:]).max() > 1e-6

@@ -349,3 +349,36 @@ def test_step_argument_errors():
         ctx.qsr_set_launch_shape(0, 3, 0)
     assert not S.theta[:, :w.P].any()                      # failed calls wrote nothing
     ctx.close()
+
+
+@pytest.mark.parametrize("opt", [W.OPT_SGDM, W.OPT_ADAMW])
+def test_per_tensor_weight_decay_table(opt):
+    """A tensor table with factors 1, 0, 0.5, 2 on the weight decay (tensor ends multiples of 4, the last one ragged)."""
+    ends = np.array([400, 404, 2000, 3003], np.int64)
+    scales = np.array([1.0, 0.0, 0.5, 2.0], np.float32)
+    w = W.tiny_workload(opt, K=3, P=3003, T=40, weight_decay=0.1)
+    lam, ths, lam_d, ths_d = G.device_inputs(w)
+    S = G.Slabs(w)
+    ctx = G.make_context(w, S, lam_d, ths_d)
+    ctx.qsr_set_tensor_table(torch.from_numpy(ends).cuda(), torch.from_numpy(scales).cuda())
+    st, H = ctx.qsr_run()
+    torch.cuda.synchronize()
+    per_coord = np.repeat(scales.astype(np.float64), np.diff(np.concatenate([[0], ends])))
+    orc = O.State(w, lam, ths, wd_scale=per_coord)
+    ost, oH = orc.run()
+    assert np.array_equal(st, ost) and np.array_equal(H, oH)
+    got = S.theta[0, :w.P].cpu().numpy()
+    assert G.rel_err(got, orc.theta[0]) <= G.REL_TOL
+    plain = G.oracle_on(w, lam, ths)
+    plain.run()
+    assert G.rel_err(got, plain.theta[0]) > 1e-4          # the table does change the result
+    # clearing the table restores the uniform weight decay
+    S2 = G.Slabs(w)
+    ctx2 = G.make_context(w, S2, lam_d, ths_d)
+    ctx2.qsr_set_tensor_table(torch.from_numpy(ends).cuda(), torch.from_numpy(scales).cuda())
+    ctx2.qsr_set_tensor_table(None, None)
+    ctx2.qsr_run()
+    torch.cuda.synchronize()
+    assert G.rel_err(S2.theta[0, :w.P].cpu().numpy(), plain.theta[0]) <= G.REL_TOL
+    ctx.close()
+    ctx2.close()
