@@ -137,6 +137,16 @@ int64_t qsr_round_length(const qsr_ctx *ctx, int64_t t);
  * breaks these rules is not detected. */
 int qsr_set_tensor_table(qsr_ctx *ctx, int32_t n_tensors, const int64_t *tensor_end_dev, const float *wd_scale_dev);
 
+/* Gradient clipping by global norm (App. C.2: threshold 1 for parallel AdamW, 4 for Local AdamW with constant H under
+ * linear decay, off in the QSR runs), in the form of the paper's software: before OPT each worker's gradient is scaled
+ * by min(1, max_norm / (||g||_2 + 1e-6)), the norm over all P coordinates of that worker (for qsr_parallel_step: of the
+ * averaged gradient).  While it is on, every step launches two more kernels first: per-worker partial sums of g^2
+ * (generated gradients are recomputed, not stored) and the K factors.  workspace_dev: caller-owned device memory of
+ * qsr_clip_workspace_floats(ctx) floats, 16-byte aligned, borrowed until clipping is switched off or the context is
+ * destroyed.  max_norm <= 0, infinite or NaN switches clipping off.  QSR_ERANGE if K exceeds 96. */
+int64_t qsr_clip_workspace_floats(const qsr_ctx *ctx);
+int qsr_set_grad_clip(qsr_ctx *ctx, double max_norm, float *workspace_dev);
+
 /* theta[k, :] <- theta0_dev[0..P) for every worker k: "each worker gets a local copy of the global iterate"
  * (Sec. 2).  Asynchronous. */
 int qsr_set_params(qsr_ctx *ctx, const float *theta0_dev);

@@ -71,6 +71,7 @@ typedef struct {
                              /* held cosine: the cosine stops decaying at t_hold (App. G)                            */
     const double *wd_scale;  /* NULL, or one factor on the weight decay per column (per-tensor weight decay; the     */
                              /* paper uses one value for the whole model, App. C)                                    */
+    double clip_norm;        /* > 0: global-norm gradient clipping threshold per worker (App. C.2); 0: off            */
 } orc_config;
 
 int orc_sizeof_real(void) { return (int)sizeof(real); }
@@ -203,29 +204,50 @@ void orc_noise_fill(uint64_t seed, int64_t k, int64_t u, int64_t i0, int64_t n, 
 /* All `rows` workers take the local step of global iteration t on the coordinates idx[0..n).
  * theta, s1, s2 are [rows, n]; row r is worker k0 + r.  idx == NULL means coordinate c is c itself.
  * grads == NULL: g = lambda*(theta - theta_star) + noise_std * z(seed, k, t, i); otherwise g = grads[r, c].
- * n_state counts the steps the optimizer state has seen before this one (bias correction uses n_state + 1). */
-void orc_local_step(const orc_config *c, int64_t rows, int64_t k0, int64_t n, const int64_t *idx,
-                    const real *lambda, const real *theta_star,
-                    real *theta, real *s1, real *s2, const real *grads,
-                    int64_t t, int64_t n_state)
+ * n_state counts the steps the optimizer state has seen before this one (bias correction uses n_state + 1).
+ * With clip_norm > 0 each worker's gradient is first scaled by min(1, clip_norm / (||g||_2 + 1e-6)), the norm taken
+ * over the n coordinates passed (gradient clipping of App. C.2, in the form of the paper's software); clipping
+ * couples the coordinates, so it is only the algorithm's clipping when all P coordinates are passed.
+ * Returns 0, or -1 if memory for one row of gradients cannot be had. */
+int orc_local_step(const orc_config *c, int64_t rows, int64_t k0, int64_t n, const int64_t *idx,
+                   const real *lambda, const real *theta_star,
+                   real *theta, real *s1, real *s2, const real *grads,
+                   int64_t t, int64_t n_state)
 {
     const real eta = (real)orc_lr(c, t);
     const real mu = (real)c->momentum;
     const real b1 = (real)c->beta1, b2 = (real)c->beta2, eps = (real)c->eps;
     const real bc1 = (real)(1.0 - pow(c->beta1, (double)(n_state + 1)));
     const real bc2 = (real)(1.0 - pow(c->beta2, (double)(n_state + 1)));
+    real *g_row = (real *)malloc((size_t)(n > 0 ? n : 1) * sizeof(real));
+    if (!g_row)
+        return -1;
     for (int64_t r = 0; r < rows; ++r) {
         const int64_t k = k0 + r;
+        /* the worker's gradient at its current parameters */
 #pragma omp parallel for schedule(static)
         for (int64_t col = 0; col < n; ++col) {
             const int64_t i = idx ? idx[col] : col;
             const int64_t e = r * n + col;
-            const real wd = (real)(c->weight_decay * (c->wd_scale ? c->wd_scale[col] : 1.0));
-            real g;
             if (grads)
-                g = grads[e];
+                g_row[col] = grads[e];
             else
-                g = lambda[col] * (theta[e] - theta_star[col]) + (real)(c->noise_std * orc_noise(c->seed, k, t, i));
+                g_row[col] = lambda[col] * (theta[e] - theta_star[col]) + (real)(c->noise_std * orc_noise(c->seed, k, t, i));
+        }
+        real clip_coef = 1;
+        if (c->clip_norm > 0.0) {
+            double sum_sq = 0.0;
+            for (int64_t col = 0; col < n; ++col)
+                sum_sq += (double)g_row[col] * (double)g_row[col];
+            double coef = c->clip_norm / (sqrt(sum_sq) + 1e-6);
+            clip_coef = (real)(coef < 1.0 ? coef : 1.0);
+        }
+        /* OPT (Eq. 1) */
+#pragma omp parallel for schedule(static)
+        for (int64_t col = 0; col < n; ++col) {
+            const int64_t e = r * n + col;
+            const real wd = (real)(c->weight_decay * (c->wd_scale ? c->wd_scale[col] : 1.0));
+            real g = clip_coef * g_row[col];
             if (c->opt == ORC_OPT_SGDM) {
                 g = g + wd * theta[e];
                 s1[e] = mu * s1[e] + g;
@@ -240,6 +262,8 @@ void orc_local_step(const orc_config *c, int64_t rows, int64_t k0, int64_t n, co
             }
         }
     }
+    free(g_row);
+    return 0;
 }
 
 /* ------------------------------------------------------------------ Algorithm 1 (Parallel OPT) */
@@ -267,9 +291,10 @@ int orc_parallel_step(const orc_config *c, int64_t K, int64_t n, const int64_t *
         }
         g_mean[col] = sum / (real)K;
     }
-    orc_local_step(c, 1, 0, n, idx, lambda, theta_star, theta, s1, s2, g_mean, t, n_state);
+    /* clipping, when on, acts on the averaged gradient, as for the paper's parallel AdamW baseline */
+    int rc = orc_local_step(c, 1, 0, n, idx, lambda, theta_star, theta, s1, s2, g_mean, t, n_state);
     free(g_mean);
-    return 0;
+    return rc;
 }
 
 /* ------------------------------------------------------------------ synchronization */
@@ -323,8 +348,9 @@ int64_t orc_run(const orc_config *c, int64_t K, int64_t n, const int64_t *idx,
     while (t < t_end) {
         int64_t H = orc_round_length(c, t);
         for (int64_t h = 0; h < H; ++h)
-            orc_local_step(c, K, 0, n, idx, lambda, theta_star, theta, s1, s2, NULL,
-                           t + h, t + h - *t_state_origin);
+            if (orc_local_step(c, K, 0, n, idx, lambda, theta_star, theta, s1, s2, NULL,
+                               t + h, t + h - *t_state_origin) != 0)
+                return -1;
         orc_sync(c, K, n, theta, s1, s2);
         if (c->state_sync == ORC_STATE_RESET)
             *t_state_origin = t + H;

@@ -33,7 +33,7 @@ class OrcConfig(C.Structure):
                 ("alpha", C.c_double), ("noise_std", C.c_double),
                 ("T", C.c_int64), ("T_warmup", C.c_int64), ("H_base", C.c_int64), ("seed", C.c_uint64),
                 ("gamma", C.c_double), ("t_switch", C.c_int64), ("t_hold", C.c_int64), ("t_period", C.c_int64),
-                ("wd_scale", C.c_void_p)]
+                ("wd_scale", C.c_void_p), ("clip_norm", C.c_double)]
 
 
 def build(force: bool = False) -> None:
@@ -71,7 +71,7 @@ def _lib(mirror: bool = False):
             lib.orc_noise.argtypes = [C.c_uint64, C.c_int64, C.c_int64, C.c_int64]
             lib.orc_noise_fill.restype = None
             lib.orc_noise_fill.argtypes = [C.c_uint64, C.c_int64, C.c_int64, C.c_int64, C.c_int64, p]
-            lib.orc_local_step.restype = None
+            lib.orc_local_step.restype = C.c_int
             lib.orc_local_step.argtypes = [cfg, C.c_int64, C.c_int64, C.c_int64, p, p, p, p, p, p, p, C.c_int64, C.c_int64]
             lib.orc_parallel_step.restype = C.c_int
             lib.orc_parallel_step.argtypes = [cfg, C.c_int64, C.c_int64, p, p, p, p, p, p, p, C.c_int64, C.c_int64]
@@ -93,7 +93,8 @@ def config_from(w) -> OrcConfig:
                      eta_max=w.eta_max, eta_min=w.eta_min, alpha=w.alpha, noise_std=w.noise_std,
                      T=w.T, T_warmup=w.T_warmup, H_base=w.H_base, seed=w.noise_seed,
                      gamma=getattr(w, "gamma", 2.0), t_switch=getattr(w, "t_switch", 0),
-                     t_hold=getattr(w, "t_hold", 0), t_period=max(1, getattr(w, "t_period", 1)))
+                     t_hold=getattr(w, "t_hold", 0), t_period=max(1, getattr(w, "t_period", 1)),
+                     clip_norm=float(getattr(w, "clip_norm", 0.0)))
 
 
 def set_threads(n: int) -> None:

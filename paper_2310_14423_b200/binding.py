@@ -26,7 +26,7 @@ QSR_OK, QSR_EINVAL, QSR_EALIGN, QSR_ECUDA, QSR_ERANGE, QSR_ESTATE = 0, -1, -2, -
 QSR_STATIC_SCRATCH_FLOATS = 1 << 20
 
 EXPORTS = ("qsr_config_check", "qsr_config_learning_rate", "qsr_config_round_length", "qsr_config_schedule",
-           "qsr_workspace_bytes", "qsr_init", "qsr_destroy", "qsr_round_length", "qsr_set_tensor_table", "qsr_set_params", "qsr_local_step",
+           "qsr_workspace_bytes", "qsr_init", "qsr_destroy", "qsr_round_length", "qsr_set_tensor_table", "qsr_clip_workspace_floats", "qsr_set_grad_clip", "qsr_set_params", "qsr_local_step",
            "qsr_local_step_sync", "qsr_parallel_step", "qsr_sync", "qsr_sync_sum_floats", "qsr_sync_partial", "qsr_sync_finish", "qsr_sync_static", "qsr_run", "qsr_launch_count",
            "qsr_set_launch_shape", "qsr_train_host", "qsr_strerror")
 
@@ -71,6 +71,8 @@ def lib():
             "qsr_destroy": (C.c_int, [vp]),
             "qsr_round_length": (i64, [vp, i64]),
             "qsr_set_tensor_table": (C.c_int, [vp, i32, vp, vp]),
+            "qsr_clip_workspace_floats": (i64, [vp]),
+            "qsr_set_grad_clip": (C.c_int, [vp, C.c_double, vp]),
             "qsr_set_params": (C.c_int, [vp, vp]),
             "qsr_local_step": (C.c_int, [vp, i64, vp]),
             "qsr_local_step_sync": (C.c_int, [vp, i64, vp, i64]),
@@ -194,6 +196,13 @@ class Context:
         n = 0 if tensor_end is None else int(tensor_end.numel())
         self._table = (tensor_end, wd_scale)
         _check(lib().qsr_set_tensor_table(self._h, n, _dptr(tensor_end), _dptr(wd_scale)), "qsr_set_tensor_table")
+
+    def qsr_clip_workspace_floats(self) -> int:
+        return int(lib().qsr_clip_workspace_floats(self._h))
+
+    def qsr_set_grad_clip(self, max_norm: float, workspace=None) -> None:
+        self._clip_ws = workspace
+        _check(lib().qsr_set_grad_clip(self._h, float(max_norm), _dptr(workspace)), "qsr_set_grad_clip")
 
     def qsr_set_params(self, theta0) -> None:
         _check(lib().qsr_set_params(self._h, _dptr(theta0)), "qsr_set_params")

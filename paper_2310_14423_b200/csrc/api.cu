@@ -20,6 +20,8 @@ struct qsr_ctx {
     int32_t n_tensors;
     const int64_t *tensor_end;
     const float *wd_scale;
+    double clip_norm;         // > 0: gradient clipping on
+    float *clip_ws;           // caller's workspace for the norm partials and the factors
 };
 
 namespace {
@@ -75,6 +77,18 @@ qsr::SyncParams sync_params(const qsr_ctx &x)
 
 int cuda_rc(int err) { return err == 0 ? QSR_OK : QSR_ECUDA; }
 
+// With clipping on: enqueue the norm pass and the factor pass for this step and make the step kernel use the factors.
+int prepare_clip(qsr_ctx &x, qsr::StepParams &p, bool parallel)
+{
+    if (!(x.clip_norm > 0.0)) return QSR_OK;
+    const int rows = parallel ? 1 : x.cfg.K;
+    const int grid = qsr::clip_grid(x.cfg.P, x.shape.step_threads);
+    x.launches += 2;
+    if (int err = qsr::launch_clip_coef(p, parallel, x.clip_norm, x.clip_ws, x.shape, x.stream)) return cuda_rc(err);
+    p.clip_coef = x.clip_ws + int64_t(grid) * rows;
+    return QSR_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -104,6 +118,7 @@ int qsr_init(qsr_ctx **out, const qsr_config *cfg, float *params, float *state1,
     x->launches = 0;
     x->partial_pending = false;
     x->n_tensors = 0; x->tensor_end = nullptr; x->wd_scale = nullptr;
+    x->clip_norm = 0.0; x->clip_ws = nullptr;
     *out = x;
     return QSR_OK;
 }
@@ -136,7 +151,8 @@ int qsr_local_step(qsr_ctx *ctx, int64_t t, const float *grads)
     if (t < 0 || t >= ctx->cfg.T || t < ctx->t_state_origin) return QSR_ERANGE;
     if (!grads && !ctx->lambda) return QSR_EINVAL;
     if (!aligned16(grads)) return QSR_EALIGN;
-    const qsr::StepParams p = step_params(*ctx, t, grads);
+    qsr::StepParams p = step_params(*ctx, t, grads);
+    if (int rc = prepare_clip(*ctx, p, false)) return rc;
     ctx->launches++;
     return cuda_rc(qsr::launch_step(p, ctx->cfg.opt, ctx->shape, ctx->stream));
 }
@@ -154,13 +170,35 @@ int qsr_set_tensor_table(qsr_ctx *ctx, int32_t n_tensors, const int64_t *tensor_
     return QSR_OK;
 }
 
+int64_t qsr_clip_workspace_floats(const qsr_ctx *ctx)
+{
+    if (!ctx) return QSR_EINVAL;
+    // partials [norm grid, K] followed by the K factors; the grid never exceeds kNormGrid whatever the block size
+    return round_up4(int64_t(qsr::kNormGrid) * ctx->cfg.K + ctx->cfg.K);
+}
+
+int qsr_set_grad_clip(qsr_ctx *ctx, double max_norm, float *workspace_dev)
+{
+    if (!ctx) return QSR_EINVAL;
+    if (!(max_norm > 0.0) || std::isinf(max_norm)) {     // off (also for NaN)
+        ctx->clip_norm = 0.0; ctx->clip_ws = nullptr;
+        return QSR_OK;
+    }
+    if (!workspace_dev) return QSR_EINVAL;
+    if (!aligned16(workspace_dev)) return QSR_EALIGN;
+    if (ctx->cfg.K > 96) return QSR_ERANGE;   // the norm pass keeps K x 128 running sums in 48 KB of shared memory
+    ctx->clip_norm = max_norm; ctx->clip_ws = workspace_dev;
+    return QSR_OK;
+}
+
 int qsr_parallel_step(qsr_ctx *ctx, int64_t t, const float *grads)
 {
     if (!ctx) return QSR_EINVAL;
     if (t < 0 || t >= ctx->cfg.T || t < ctx->t_state_origin) return QSR_ERANGE;
     if (!grads && !ctx->lambda) return QSR_EINVAL;
     if (!aligned16(grads)) return QSR_EALIGN;
-    const qsr::StepParams p = step_params(*ctx, t, grads);
+    qsr::StepParams p = step_params(*ctx, t, grads);
+    if (int rc = prepare_clip(*ctx, p, true)) return rc;
     ctx->launches++;
     return cuda_rc(qsr::launch_parallel_step(p, ctx->cfg.opt, ctx->shape, ctx->stream));
 }
@@ -176,7 +214,8 @@ int qsr_local_step_sync(qsr_ctx *ctx, int64_t t, const float *grads, int64_t t_n
     if (t < 0 || t >= ctx->cfg.T || t < ctx->t_state_origin || t_next < 0 || t_next > ctx->cfg.T) return QSR_ERANGE;
     if (!grads && !ctx->lambda) return QSR_EINVAL;
     if (!aligned16(grads)) return QSR_EALIGN;
-    const qsr::StepParams p = step_params(*ctx, t, grads);
+    qsr::StepParams p = step_params(*ctx, t, grads);
+    if (int rc = prepare_clip(*ctx, p, false)) return rc;
     ctx->launches++;
     return cuda_rc(qsr::launch_step_mean(p, ctx->cfg.opt, ctx->shape, ctx->stream));
 }

@@ -33,7 +33,10 @@ struct StepParams {
     int32_t n_tensors;             // 0: uniform weight decay
     const int64_t *tensor_end;     // device [n_tensors]: one past each tensor's last coordinate, ascending
     const float *wd_scale;         // device [n_tensors]: factor on the weight decay of each tensor
+    const float *clip_coef;        // NULL, or device [K] ([1] for Algorithm 1): gradient-clipping factor per worker
 };
+
+constexpr int kNormGrid = 1184;    // blocks of the gradient-norm pass (8 per SM on a 148-SM part)
 
 struct SyncParams {
     float *slab[3];           // arrays to average (theta first), then arrays to zero
@@ -64,6 +67,9 @@ int launch_sync_partial(const SyncParams &p, const LaunchShape &shape, void *str
 int launch_sync_finish(const SyncParams &p, const LaunchShape &shape, void *stream);   // sums -> rows (+ zero)
 int launch_broadcast(float *theta, const float *theta0, int64_t P, int64_t stride, int32_t K,
                      const LaunchShape &shape, void *stream);
+// Gradient clipping: grid of the norm pass and the two passes that leave the factors at ws + clip_grid(...) * rows.
+int clip_grid(int64_t P, int threads);
+int launch_clip_coef(const StepParams &p, bool parallel, double max_norm, float *ws, const LaunchShape &shape, void *stream);
 // Both phases through the library's own static scratch; -1 if the sums exceed QSR_STATIC_SCRATCH_FLOATS.
 int launch_sync_static(const SyncParams &p, const LaunchShape &shape, void *stream);
 

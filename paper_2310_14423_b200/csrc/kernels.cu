@@ -160,6 +160,10 @@ __global__ void local_step_kernel(const StepParams p)
                             g[r].z = fmaf(p.sigma, z.z, lam.z * (th[r].z - ths.z));
                             g[r].w = fmaf(p.sigma, z.w, lam.w * (th[r].w - ths.w));
                         }
+                        if (p.clip_coef) {   // gradient clipping: this worker's factor min(1, c / (||g|| + 1e-6))
+                            const float cs = __ldg(p.clip_coef + k + r);
+                            g[r].x *= cs; g[r].y *= cs; g[r].z *= cs; g[r].w *= cs;
+                        }
                         opt_update<OPT>(th[r].x, a[r].x, b[r].x, g[r].x, p, wdv);
                         opt_update<OPT>(th[r].y, a[r].y, b[r].y, g[r].y, p, wdv);
                         opt_update<OPT>(th[r].z, a[r].z, b[r].z, g[r].z, p, wdv);
@@ -192,6 +196,7 @@ __global__ void local_step_kernel(const StepParams p)
                         const float zc = c == 0 ? z.x : (c == 1 ? z.y : z.z);
                         g = fmaf(p.sigma, zc, p.lambda[i] * (th - p.theta_star[i]));
                     }
+                    if (p.clip_coef) g *= __ldg(p.clip_coef + k);
                     opt_update<OPT>(th, a, b, g, p, wdv);
                     if (FUSE_MEAN) acc += th;
                     else p.theta[e] = th;
@@ -256,7 +261,11 @@ __global__ void parallel_step_kernel(const StepParams p)
                     sum.w += fmaf(p.sigma, z.w, pull.w);
                 }
             }
-            const float4 g = div4(sum, Kf);
+            float4 g = div4(sum, Kf);
+            if (p.clip_coef) {   // clipping acts on the averaged gradient
+                const float cs = __ldg(p.clip_coef);
+                g.x *= cs; g.y *= cs; g.z *= cs; g.w *= cs;
+            }
             opt_update<OPT>(th.x, a.x, b.x, g.x, p, wdv);
             opt_update<OPT>(th.y, a.y, b.y, g.y, p, wdv);
             opt_update<OPT>(th.z, a.z, b.z, g.z, p, wdv);
@@ -278,11 +287,93 @@ __global__ void parallel_step_kernel(const StepParams p)
                         sum += fmaf(p.sigma, zc, p.lambda[i] * (th - p.theta_star[i]));
                     }
                 }
-                opt_update<OPT>(th, a, b, sum / Kf, p, wdv);
+                float g = sum / Kf;
+                if (p.clip_coef) g *= __ldg(p.clip_coef);
+                opt_update<OPT>(th, a, b, g, p, wdv);
                 p.theta[i] = th;
                 p.s1[i] = a;
                 if (OPT == QSR_OPT_ADAMW) p.s2[i] = b;
             }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------- gradient clipping
+
+// Pass 1 of global-norm clipping (App. C.2): partial sums of g^2, per worker (PARALLEL = false: one sum per row k of
+// the gradient that worker's step will use) or of the averaged gradient (PARALLEL = true: Algorithm 1).  Generated
+// gradients are recomputed here with the very expressions of the step kernel -- the noise is a pure function of
+// (seed, worker, step, coordinate) -- so nothing has to be stored: the pass reads theta once (4 B per update).
+// The grid is fixed (kNormGrid blocks at most) so that the partials fit a small workspace; a thread strides over
+// columns and keeps its running sum for worker k in shared memory at acc[k * blockDim.x + threadIdx.x].
+// partial is [gridDim.x, rows] with rows = PARALLEL ? 1 : K.  Summation order is fixed: results are deterministic.
+// 16-byte load when the whole column lies inside the row, scalar loads (zeros beyond P) for the ragged last column.
+__device__ __forceinline__ float4 ld4_guarded(const float *q, int valid)
+{
+    if (valid == 4) return ld4(q);
+    return make_float4(q[0], valid > 1 ? q[1] : 0.f, valid > 2 ? q[2] : 0.f, 0.f);
+}
+
+template <bool EXT_GRAD, bool PARALLEL>
+__global__ void grad_sqnorm_kernel(const StepParams p, float *partial)
+{
+    extern __shared__ float acc[];
+    const int rows = PARALLEL ? 1 : p.K;
+    for (int r = 0; r < rows; ++r) acc[r * blockDim.x + threadIdx.x] = 0.f;
+    const int64_t n_col = (p.P + 3) >> 2;
+    const int64_t grid_stride = int64_t(gridDim.x) * blockDim.x;
+    const float Kf = float(p.K);
+    for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < n_col; j += grid_stride) {
+        const int64_t i0 = j << 2;
+        const int valid = i0 + 4 <= p.P ? 4 : int(p.P - i0);
+        float4 lam = make_float4(0.f, 0.f, 0.f, 0.f), ths = lam, sum = lam;
+        if (!EXT_GRAD) {
+            lam = ld4_guarded(p.lambda + i0, valid);     // zero lambda and zero noise weight make the lanes beyond P vanish
+            ths = ld4_guarded(p.theta_star + i0, valid);
+        }
+        for (int k = 0; k < p.K; ++k) {
+            float4 g;
+            if (EXT_GRAD) {
+                g = ld4_guarded(p.grads + int64_t(k) * p.stride + i0, valid);
+            } else {
+                // Algorithm 1 evaluates every worker's gradient at the single model in row 0
+                const float4 th = ld4_guarded(p.theta + int64_t(PARALLEL ? 0 : k) * p.stride + i0, valid);
+                const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.key0, p.key1);
+                g.x = fmaf(p.sigma, z.x, lam.x * (th.x - ths.x));
+                g.y = valid > 1 ? fmaf(p.sigma, z.y, lam.y * (th.y - ths.y)) : 0.f;
+                g.z = valid > 2 ? fmaf(p.sigma, z.z, lam.z * (th.z - ths.z)) : 0.f;
+                g.w = valid > 3 ? fmaf(p.sigma, z.w, lam.w * (th.w - ths.w)) : 0.f;
+            }
+            if (PARALLEL) sum = add4(sum, g);
+            else acc[k * blockDim.x + threadIdx.x] += (g.x * g.x + g.y * g.y) + (g.z * g.z + g.w * g.w);
+        }
+        if (PARALLEL) {
+            sum = div4(sum, Kf);
+            acc[threadIdx.x] += (sum.x * sum.x + sum.y * sum.y) + (sum.z * sum.z + sum.w * sum.w);
+        }
+    }
+    __syncthreads();
+    // block reduction per worker: warp w folds rows w, w + n_warps, ...
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    for (int r = warp; r < rows; r += n_warps) {
+        float v = 0.f;
+        for (int t = lane; t < int(blockDim.x); t += 32) v += acc[r * blockDim.x + t];
+        for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) partial[int64_t(blockIdx.x) * rows + r] = v;
+    }
+}
+
+// Pass 2: coef[r] = min(1, max_norm / (sqrt(sum of partials) + 1e-6)), accumulated in binary64 in a fixed order.
+__global__ void clip_coef_kernel(const float *partial, int n_blocks, int rows, double max_norm, float *coef)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    for (int r = warp; r < rows; r += n_warps) {
+        double s = 0.0;
+        for (int b = lane; b < n_blocks; b += 32) s += double(partial[int64_t(b) * rows + r]);
+        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) {
+            const double c = max_norm / (sqrt(s) + 1e-6);
+            coef[r] = float(c < 1.0 ? c : 1.0);
         }
     }
 }
@@ -429,6 +520,34 @@ int launch_parallel_step(const StepParams &p, int opt, const LaunchShape &shape,
         if (ext) parallel_step_kernel<QSR_OPT_ADAMW, true><<<grid, shape.step_threads, 0, st>>>(p);
         else parallel_step_kernel<QSR_OPT_ADAMW, false><<<grid, shape.step_threads, 0, st>>>(p);
     }
+    return int(cudaGetLastError());
+}
+
+int clip_grid(int64_t P, int threads)
+{
+    const int64_t want = (((P + 3) >> 2) + threads - 1) / threads;
+    return int(want < kNormGrid ? (want < 1 ? 1 : want) : kNormGrid);
+}
+
+// Enqueues the two clipping passes; afterwards ws[clip_grid*rows .. +rows) holds the factors.
+int launch_clip_coef(const StepParams &p, bool parallel, double max_norm, float *ws, const LaunchShape &shape, void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int threads = shape.step_threads;
+    const int rows = parallel ? 1 : p.K;
+    const int grid = clip_grid(p.P, threads);
+    const size_t smem = size_t(rows) * threads * sizeof(float);
+    if (smem > 48 * 1024) return int(cudaErrorInvalidValue);
+    const bool ext = p.grads != nullptr;
+    if (parallel) {
+        if (ext) grad_sqnorm_kernel<true, true><<<grid, threads, smem, st>>>(p, ws);
+        else grad_sqnorm_kernel<false, true><<<grid, threads, smem, st>>>(p, ws);
+    } else {
+        if (ext) grad_sqnorm_kernel<true, false><<<grid, threads, smem, st>>>(p, ws);
+        else grad_sqnorm_kernel<false, false><<<grid, threads, smem, st>>>(p, ws);
+    }
+    if (cudaError_t e = cudaGetLastError()) return int(e);
+    clip_coef_kernel<<<1, 256, 0, st>>>(ws, grid, rows, max_norm, ws + int64_t(grid) * rows);
     return int(cudaGetLastError());
 }
 

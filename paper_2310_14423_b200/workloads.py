@@ -167,6 +167,7 @@ class Workload:
     t_switch: int = 0           # switching step of the post-local and SWAP schedules
     t_hold: int = 0             # halving / held-cosine schedules: last step at the regular value
     t_period: int = 1           # halving schedule: steps between halvings
+    clip_norm: float = 0.0      # > 0: per-worker global-norm gradient clipping threshold (App. C.2); 0: off
 
     @property
     def P(self) -> int:

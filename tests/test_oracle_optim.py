@@ -405,3 +405,57 @@ def test_per_tensor_weight_decay_equals_torch_param_groups():
         plain = O.State(w, lam, ths)
         plain.run()
         assert np.abs(plain.theta[0, 8:] - S.theta[0, 8:]).max() > 1e-6
+
+
+# ------------------------------------------------------------------ gradient clipping (App. C.2)
+
+def test_clipped_single_worker_equals_torch_clip_grad_norm():
+    for opt in (W.OPT_SGDM, W.OPT_ADAMW):
+        w = W.tiny_workload(opt, K=1, P=18, T=30, clip_norm=0.35, noise_std=0.3)
+        lam, ths = _inputs(w)
+        lam, ths = lam.astype(np.float64), ths.astype(np.float64)
+        S = O.State(w, lam, ths)
+        S.run()
+        p = torch.zeros(18, dtype=torch.float64, requires_grad=True)
+        topt = (torch.optim.SGD([p], lr=1.0, momentum=w.momentum, weight_decay=w.weight_decay) if opt == W.OPT_SGDM
+                else torch.optim.AdamW([p], lr=1.0, betas=(w.beta1, w.beta2), eps=w.eps, weight_decay=w.weight_decay))
+        clipped = 0
+        for t in range(w.T):
+            for g in topt.param_groups:
+                g["lr"] = 0.5 * w.eta_max * (1 + math.cos(math.pi * t / w.T))
+            p.grad = torch.from_numpy(_grad(w, lam, ths, p.detach().numpy(), 0, t))
+            clipped += float(torch.nn.utils.clip_grad_norm_([p], 0.35)) > 0.35
+            topt.step()
+        assert 0 < clipped                                  # the threshold did bite
+        np.testing.assert_allclose(S.theta[0], p.detach().numpy(), rtol=1e-10, atol=1e-13)
+        free = O.State(w.replace(clip_norm=0.0), lam, ths)
+        free.run()
+        assert np.abs(free.theta[0] - S.theta[0]).max() > 1e-4
+
+
+def test_clipping_closed_form_and_inactive_threshold():
+    """Plain SGD on a constant gradient g with ||g|| > c: every step moves by eta_t * c * g / (||g|| + 1e-6)."""
+    w = W.tiny_workload(W.OPT_SGDM, K=2, P=4, T=10, momentum=0.0, weight_decay=0.0, sched=W.SCHED_CONST, eta_max=0.1,
+                        clip_norm=0.5, rule=W.RULE_CONST_H, H_base=10)
+    g = np.array([3.0, -4.0, 0.0, 12.0])                  # norm 13
+    S = O.State(w, np.zeros(4), np.zeros(4))
+    for t in range(w.T):
+        S.local_step(t, grads=np.tile(g, (2, 1)))
+    np.testing.assert_allclose(S.theta[0], -10 * 0.1 * 0.5 * g / (13.0 + 1e-6), rtol=1e-12)
+    # a threshold above every gradient norm changes nothing
+    a = W.tiny_workload(W.OPT_ADAMW, K=3, P=15, T=20)
+    lam, ths = _inputs(a)
+    x, y = O.State(a, lam, ths), O.State(a.replace(clip_norm=1e6), lam, ths)
+    x.run(), y.run()
+    assert np.array_equal(x.theta, y.theta)
+
+
+def test_clipping_is_per_worker():
+    """Each worker clips by its own gradient norm: a worker with a small gradient is left alone."""
+    w = W.tiny_workload(W.OPT_SGDM, K=2, P=3, T=5, momentum=0.0, weight_decay=0.0, sched=W.SCHED_CONST, eta_max=1.0,
+                        clip_norm=1.0)
+    S = O.State(w, np.zeros(3), np.zeros(3))
+    g = np.array([[0.3, 0.0, 0.4], [30.0, 0.0, 40.0]])   # norms 0.5 and 50
+    S.local_step(0, grads=g)
+    np.testing.assert_allclose(S.theta[0], -g[0], rtol=1e-13)
+    np.testing.assert_allclose(S.theta[1], -g[1] / (50.0 + 1e-6), rtol=1e-13)

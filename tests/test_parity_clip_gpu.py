@@ -1,0 +1,108 @@
+"""GPU parity for gradient clipping by global norm (App. C.2): Local OPT with per-worker clipping and Algorithm 1
+with the averaged gradient clipped, against the oracle on ALL coordinates (clipping couples them, so there is no
+coordinate subset here)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import qsr_oracle as O
+from paper_2310_14423_b200 import binding as B
+from paper_2310_14423_b200 import workloads as W
+
+import gpu_harness as G
+
+pytestmark = pytest.mark.gpu
+
+
+def _clip_context(w, S, lam_d, ths_d):
+    ctx = G.make_context(w, S, lam_d, ths_d)
+    ws = torch.full((ctx.qsr_clip_workspace_floats() + 8,), 7.0, device="cuda")
+    ctx.qsr_set_grad_clip(w.clip_norm, ws)
+    return ctx, ws
+
+
+@pytest.mark.parametrize("opt", [W.OPT_SGDM, W.OPT_ADAMW])
+@pytest.mark.parametrize("K,P", [(1, 3), (3, 1001), (16, 40002), (5, 300000)])
+def test_clipped_local_runs(opt, K, P):
+    # the threshold sits inside the range of gradient norms of the run, so some steps clip and some do not
+    clip = {3: 0.3, 1001: 3.0, 40002: 20.0, 300000: 55.0}[P]
+    w = W.tiny_workload(opt, K=K, P=P, T=30, clip_norm=clip)
+    lam, ths, lam_d, ths_d = G.device_inputs(w)
+    S = G.Slabs(w)
+    ctx, ws = _clip_context(w, S, lam_d, ths_d)
+    st, H = ctx.qsr_run()
+    torch.cuda.synchronize()
+    assert ctx.qsr_launch_count() == 3 * w.T              # norm pass, factor pass, step
+    orc = G.oracle_on(w, lam, ths)
+    ost, oH = orc.run()
+    assert np.array_equal(st, ost) and np.array_equal(H, oH)
+    assert G.rel_err(S.theta[:, :P].cpu().numpy(), orc.theta) <= G.REL_TOL
+    free = G.oracle_on(w.replace(clip_norm=0.0), lam, ths)
+    free.run()
+    assert G.rel_err(S.theta[0, :P].cpu().numpy(), free.theta[0]) > 1e-4   # clipping did change the run
+    assert S.guards_intact() and bool((ws[-8:] == 7.0).all())
+    ctx.close()
+
+
+def test_clip_factors_against_numpy():
+    """The factors themselves, for gradients from a slab: min(1, c / (||g_k|| + 1e-6)) per worker."""
+    K, P = 6, 123457
+    w = W.tiny_workload(W.OPT_SGDM, K=K, P=P, T=5, momentum=0.0, weight_decay=0.0, sched=W.SCHED_CONST, eta_max=1.0,
+                        clip_norm=100.0)
+    S = G.Slabs(w, n_extra=1)
+    ctx = G.make_context(w, S, None, None)
+    ws = torch.zeros(ctx.qsr_clip_workspace_floats(), device="cuda")
+    ctx.qsr_set_grad_clip(w.clip_norm, ws)
+    grads = S.extra[0]
+    scale = torch.tensor([0.01, 0.1, 0.28, 0.3, 1.0, 10.0], device="cuda").view(K, 1)
+    grads[:, :P] = torch.randn(K, P, device="cuda") * scale
+    ctx.qsr_local_step(0, grads)
+    torch.cuda.synchronize()
+    g = grads[:, :P].double().cpu().numpy()
+    coef = np.minimum(1.0, 100.0 / (np.sqrt((g * g).sum(axis=1)) + 1e-6))
+    assert (coef < 1).any() and (coef == 1).any()
+    theta = S.theta[:, :P].double().cpu().numpy()
+    np.testing.assert_allclose(theta, -coef[:, None] * g, rtol=2e-6, atol=1e-9)
+    ctx.close()
+
+
+@pytest.mark.parametrize("opt", [W.OPT_SGDM, W.OPT_ADAMW])
+def test_clipped_parallel_steps(opt):
+    K, P = 8, 50003
+    w = W.tiny_workload(opt, K=K, P=P, T=30, clip_norm=12.0)
+    lam, ths, lam_d, ths_d = G.device_inputs(w)
+    S = G.Slabs(w)
+    ctx, ws = _clip_context(w, S, lam_d, ths_d)
+    orc = O.State(w, lam, ths, rows=1)
+    for t in range(w.T):
+        ctx.qsr_parallel_step(t)
+        orc.parallel_step(t, K)
+    torch.cuda.synchronize()
+    assert G.rel_err(S.theta[0, :P].cpu().numpy(), orc.theta[0]) <= G.REL_TOL
+    free = O.State(w.replace(clip_norm=0.0), lam, ths, rows=1)
+    for t in range(w.T):
+        free.parallel_step(t, K)
+    assert G.rel_err(S.theta[0, :P].cpu().numpy(), free.theta[0]) > 1e-4
+    ctx.close()
+
+
+def test_clip_switch_and_argument_errors():
+    w = W.tiny_workload(W.OPT_SGDM, K=2, P=64, T=10)
+    lam, ths, lam_d, ths_d = G.device_inputs(w)
+    S = G.Slabs(w)
+    ctx = G.make_context(w, S, lam_d, ths_d)
+    with pytest.raises(B.QsrError) as e:
+        ctx.qsr_set_grad_clip(1.0, None)
+    assert e.value.status == B.QSR_EINVAL
+    ws = torch.zeros(ctx.qsr_clip_workspace_floats() + 4, device="cuda")
+    with pytest.raises(B.QsrError) as e:
+        ctx.qsr_set_grad_clip(1.0, ws[1:])
+    assert e.value.status == B.QSR_EALIGN
+    ctx.qsr_set_grad_clip(1.0, ws)
+    ctx.qsr_local_step(0)
+    assert ctx.qsr_launch_count() == 3
+    ctx.qsr_set_grad_clip(0.0)                # off again
+    ctx.qsr_local_step(1)
+    assert ctx.qsr_launch_count() == 4
+    torch.cuda.synchronize()
+    ctx.close()
