@@ -60,6 +60,26 @@ def test_noise_matches_oracle_elementwise():
     ctx.close()
 
 
+def test_noise_has_no_bias_against_oracle():
+    """4 M normals: the fp32 generator's error against the binary64 oracle is rounding-sized and averages out.
+    A bias b in the noise would shift a coordinate of curvature lambda by sigma*b/lambda, so it is bounded tightly."""
+    P, K, t = 1 << 20, 4, 4242
+    w = W.tiny_workload(W.OPT_SGDM, K=K, P=P, T=5000, sched=W.SCHED_CONST, eta_max=1.0, momentum=0.0,
+                        weight_decay=0.0, noise_std=1.0)
+    S = G.Slabs(w)
+    zero = torch.zeros(P, device="cuda")
+    ctx = G.make_context(w, S, zero, zero)
+    ctx.qsr_local_step(t)
+    torch.cuda.synchronize()
+    z_gpu = -S.theta[:, :P].cpu().numpy().astype(np.float64)
+    err = np.concatenate([z_gpu[k] - O.noise_fill(w.noise_seed, k, t, 0, P) for k in range(K)])
+    assert np.abs(err).max() < 2e-6
+    assert np.sqrt(np.mean(err * err)) < 1.5e-7
+    assert abs(err.mean()) < 2e-9
+    assert abs(z_gpu.mean()) < 4 / np.sqrt(K * P) and abs(z_gpu.var() - 1) < 6 / np.sqrt(K * P)
+    ctx.close()
+
+
 def test_noise_high_counter_words():
     """Worker offset, a step beyond 2^16 and the last coordinates of a long row reach the counter unchanged."""
     P = 1 << 16
