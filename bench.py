@@ -43,8 +43,8 @@ FALLBACK_HBM_GBS = 6650.0
 # once, so traffic grows in proportion to K*P).  Valid only for the kernel source it was taken from: the hash covers
 # the noise generator, the optimizer update and local_step_kernel in csrc/kernels.cu.
 NCU_TRAFFIC = {
-    "step_source_sha256": "eff7b805a4e9d29a8d1fddd775f0803c9dd528bb49ecc555ef184563b06a504e",
-    "bytes_per_update": {"adamw": 24.077, "sgdm": 16.076},
+    "step_source_sha256": "bf4023c4b1c52a79baf4977b409ea2f8f6fbf8b2f3bdf9a0bfdafcffbe5e8d66",
+    "bytes_per_update": {"adamw": 24.068, "sgdm": 16.069},
 }
 
 
