@@ -286,15 +286,19 @@ def main():
             n_ev += 1
             kinds.append("sync")
             continue
+        if t + 1 in ends:
+            # sharded round end: last step fused with this rank's row sums, all-reduce, finish
+            ctx.qsr_local_step_partial(t, sums)
+            all_reduce(sums[:ctx.qsr_sync_sum_floats()])
+            ctx.qsr_sync_finish(sums, K_total, t + 1)
+            ev[n_ev].record()
+            n_ev += 1
+            kinds.append("sync")
+            continue
         ctx.qsr_local_step(t)
         ev[n_ev].record()
         n_ev += 1
         kinds.append("step")
-        if t + 1 in ends:
-            do_sync(ctx, t + 1)
-            ev[n_ev].record()
-            n_ev += 1
-            kinds.append("sync")
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
@@ -406,10 +410,12 @@ def main():
                            "frac_of_measured": sa_gbs / peak, "frac_of_nominal_8TBps": sa_gbs / NOMINAL_HBM_GBS,
                            "note": "stand-alone replica-mean kernel (used when the state is averaged or reset)"}
     if sync_ms is not None and sharded_path:
-        sync_bytes = 8.0 * K_local * w.P + 8.0 * w.P
-        sync_gbs = sync_bytes / (sync_ms * 1e-3) / 1e9
-        kernels["sync"] = {"launches": n_syncs, "avg_ms": sync_ms, "GBps": sync_gbs, "frac_of_measured": sync_gbs / peak,
-                           "note": "partial kernel + NCCL all-reduce + finish kernel"}
+        # last step without the theta write-back, [P] sums out, then sums in and K rows written
+        end_bytes = step_bytes - 4.0 * K_local * w.P + 8.0 * w.P + 4.0 * K_local * w.P
+        end_gbs = end_bytes / (sync_ms * 1e-3) / 1e9
+        kernels["sharded_round_end"] = {"launches": n_syncs, "avg_ms": sync_ms, "GBps": end_gbs,
+                                        "frac_of_measured": end_gbs / peak,
+                                        "note": "last step fused with row sums + NCCL all-reduce of P floats + finish kernel"}
 
     label = {"c4": "c4: ViT-B/16-shaped parameter set, Local AdamW + QSR",
              "c3": "c3: ResNet-152-shaped parameter set, Local SGD + QSR"}.get(w.name, w.name)

@@ -183,6 +183,11 @@ int qsr_parallel_step(qsr_ctx *ctx, int64_t t, const float *grads);
  * `sum` holds qsr_sync_sum_floats(ctx) floats. */
 int64_t qsr_sync_sum_floats(const qsr_ctx *ctx);
 int qsr_sync_partial(qsr_ctx *ctx, float *sum);
+/* The round's last local step fused with qsr_sync_partial (state_sync = QSR_STATE_KEEP; otherwise the two launches are
+ * issued): the kernel writes the row sums of the NEW parameters to `sum` and does not write the parameter rows at all
+ * -- qsr_sync_finish overwrites every row with the global mean anyway -- so a sharded round end costs 4 B per update
+ * less than a plain step.  After this call the parameter slab holds the pre-step values until qsr_sync_finish runs. */
+int qsr_local_step_partial(qsr_ctx *ctx, int64_t t, const float *grads, float *sum);
 int qsr_sync_finish(qsr_ctx *ctx, const float *sum, int32_t K_total, int64_t t_next);
 
 /* A synchronization for callers that have no device buffer to spare and may not create one.  The paper has no

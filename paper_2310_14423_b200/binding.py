@@ -27,7 +27,7 @@ QSR_STATIC_SCRATCH_FLOATS = 1 << 20
 
 EXPORTS = ("qsr_config_check", "qsr_config_learning_rate", "qsr_config_round_length", "qsr_config_schedule",
            "qsr_workspace_bytes", "qsr_init", "qsr_destroy", "qsr_round_length", "qsr_set_tensor_table", "qsr_clip_workspace_floats", "qsr_set_grad_clip", "qsr_set_params", "qsr_local_step",
-           "qsr_local_step_sync", "qsr_parallel_step", "qsr_sync", "qsr_sync_sum_floats", "qsr_sync_partial", "qsr_sync_finish", "qsr_sync_static", "qsr_run", "qsr_launch_count",
+           "qsr_local_step_sync", "qsr_parallel_step", "qsr_sync", "qsr_sync_sum_floats", "qsr_sync_partial", "qsr_local_step_partial", "qsr_sync_finish", "qsr_sync_static", "qsr_run", "qsr_launch_count",
            "qsr_set_launch_shape", "qsr_train_host", "qsr_strerror")
 
 
@@ -80,6 +80,7 @@ def lib():
             "qsr_sync": (C.c_int, [vp, i64]),
             "qsr_sync_sum_floats": (i64, [vp]),
             "qsr_sync_partial": (C.c_int, [vp, vp]),
+            "qsr_local_step_partial": (C.c_int, [vp, i64, vp, vp]),
             "qsr_sync_finish": (C.c_int, [vp, vp, i32, i64]),
             "qsr_sync_static": (C.c_int, [vp, i64]),
             "qsr_run": (C.c_int, [vp, i64, i64, vp, vp, i64, C.POINTER(i64)]),
@@ -224,6 +225,9 @@ class Context:
 
     def qsr_sync_partial(self, sums) -> None:
         _check(lib().qsr_sync_partial(self._h, _dptr(sums)), "qsr_sync_partial")
+
+    def qsr_local_step_partial(self, t: int, sums, grads=None) -> None:
+        _check(lib().qsr_local_step_partial(self._h, int(t), _dptr(grads), _dptr(sums)), "qsr_local_step_partial")
 
     def qsr_sync_finish(self, sums, K_total: int, t_next: int) -> None:
         _check(lib().qsr_sync_finish(self._h, _dptr(sums), int(K_total), int(t_next)), "qsr_sync_finish")

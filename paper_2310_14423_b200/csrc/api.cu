@@ -231,6 +231,27 @@ int qsr_sync(qsr_ctx *ctx, int64_t t_next)
     return rc;
 }
 
+int qsr_local_step_partial(qsr_ctx *ctx, int64_t t, const float *grads, float *sum)
+{
+    if (!ctx || !sum) return QSR_EINVAL;
+    if (!aligned16(sum)) return QSR_EALIGN;
+    if (ctx->cfg.state_sync != QSR_STATE_KEEP) {
+        // the state slabs need their own sums (AVERAGE) or nothing fused is gained (RESET): two launches
+        if (int rc = qsr_local_step(ctx, t, grads)) return rc;
+        return qsr_sync_partial(ctx, sum);
+    }
+    if (t < 0 || t >= ctx->cfg.T || t < ctx->t_state_origin) return QSR_ERANGE;
+    if (!grads && !ctx->lambda) return QSR_EINVAL;
+    if (!aligned16(grads)) return QSR_EALIGN;
+    qsr::StepParams p = step_params(*ctx, t, grads);
+    if (int rc = prepare_clip(*ctx, p, false)) return rc;
+    p.sum_out = sum;
+    ctx->launches++;
+    const int rc = cuda_rc(qsr::launch_step_sum(p, ctx->cfg.opt, ctx->shape, ctx->stream));
+    if (rc == QSR_OK) ctx->partial_pending = true;
+    return rc;
+}
+
 int64_t qsr_sync_sum_floats(const qsr_ctx *ctx)
 {
     if (!ctx) return QSR_EINVAL;

@@ -34,6 +34,7 @@ struct StepParams {
     const int64_t *tensor_end;     // device [n_tensors]: one past each tensor's last coordinate, ascending
     const float *wd_scale;         // device [n_tensors]: factor on the weight decay of each tensor
     const float *clip_coef;        // NULL, or device [K] ([1] for Algorithm 1): gradient-clipping factor per worker
+    float *sum_out;                // step fused with the partial sums of a sharded synchronization: device [P4]
 };
 
 constexpr int kNormGrid = 1184;    // blocks of the gradient-norm pass (8 per SM on a 148-SM part)
@@ -61,6 +62,7 @@ struct LaunchShape {
 // kernels.cu -- each returns a cudaError_t cast to int (0 = success) after enqueueing one kernel.
 int launch_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream);
 int launch_step_mean(const StepParams &p, int opt, const LaunchShape &shape, void *stream);   // step + replica mean
+int launch_step_sum(const StepParams &p, int opt, const LaunchShape &shape, void *stream);    // step + row sums to p.sum_out
 int launch_parallel_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream);  // Algorithm 1, row 0
 int launch_sync(const SyncParams &p, const LaunchShape &shape, void *stream);          // mean + write back (+ zero)
 int launch_sync_partial(const SyncParams &p, const LaunchShape &shape, void *stream);  // sums only

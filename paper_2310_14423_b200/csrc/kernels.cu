@@ -115,14 +115,18 @@ __device__ __forceinline__ void st4(float *p, float4 v) { *reinterpret_cast<floa
 __device__ __forceinline__ float4 add4(float4 x, float4 y) { return make_float4(x.x + y.x, x.y + y.y, x.z + y.z, x.w + y.w); }
 __device__ __forceinline__ float4 div4(float4 x, float d) { return make_float4(x.x / d, x.y / d, x.z / d, x.w / d); }
 
-// One local step of all K workers.  With FUSE_MEAN the step is the last of its round and the kernel also ends the
+// One local step of all K workers.  With FUSE != 0 the step is the last of its round and the kernel also ends the
 // round (Algorithm 2's averaging, state kept per worker): the thread that owns a column sees every worker's new
 // parameters anyway, so it sums them as it goes (k ascending, fp32: the order of the stand-alone sync kernel, hence
-// the same bits) and writes the mean to all K rows instead of the K different values.  The averaging then costs no
-// HBM traffic at all: theta is read once and written once, exactly as in a plain step.
+// the same bits).  FUSE_MEAN writes the mean to all K rows instead of the K different values: the averaging then
+// costs no HBM traffic at all, theta is read once and written once exactly as in a plain step.  FUSE_SUM is the
+// multi-GPU form: the column's sum goes to p.sum_out (the buffer that is all-reduced over processes) and theta is not
+// written at all, since the finish kernel will overwrite every row with the global mean.
 // No launch bound: the register count decides how many threads fit; a block shape that does not fit is
 // reported by the launch as an error, not silently spilled.
-template <int OPT, bool EXT_GRAD, int ROWS, bool FUSE_MEAN>
+enum { FUSE_NONE = 0, FUSE_MEAN = 1, FUSE_SUM = 2 };
+
+template <int OPT, bool EXT_GRAD, int ROWS, int FUSE>
 __global__ void local_step_kernel(const StepParams p)
 {
     const int64_t n_col = (p.P + 3) >> 2;
@@ -168,17 +172,19 @@ __global__ void local_step_kernel(const StepParams p)
                         opt_update<OPT>(th[r].y, a[r].y, b[r].y, g[r].y, p, wdv);
                         opt_update<OPT>(th[r].z, a[r].z, b[r].z, g[r].z, p, wdv);
                         opt_update<OPT>(th[r].w, a[r].w, b[r].w, g[r].w, p, wdv);
-                        if (FUSE_MEAN) acc = add4(acc, th[r]);
+                        if (FUSE != FUSE_NONE) acc = add4(acc, th[r]);
                         else st4(p.theta + e, th[r]);
                         st4(p.s1 + e, a[r]);
                         if (OPT == QSR_OPT_ADAMW) st4(p.s2 + e, b[r]);
                     }
                 }
             }
-            if (FUSE_MEAN) {
+            if (FUSE == FUSE_MEAN) {
                 const float4 mean = div4(acc, float(p.K));
 #pragma unroll 4
                 for (int k = 0; k < p.K; ++k) st4(p.theta + int64_t(k) * p.stride + i0, mean);
+            } else if (FUSE == FUSE_SUM) {
+                st4(p.sum_out + i0, acc);
             }
         } else {
             // Ragged last column: P is not a multiple of 4.  Scalar accesses, nothing beyond P is touched.
@@ -198,14 +204,16 @@ __global__ void local_step_kernel(const StepParams p)
                     }
                     if (p.clip_coef) g *= __ldg(p.clip_coef + k);
                     opt_update<OPT>(th, a, b, g, p, wdv);
-                    if (FUSE_MEAN) acc += th;
+                    if (FUSE != FUSE_NONE) acc += th;
                     else p.theta[e] = th;
                     p.s1[e] = a;
                     if (OPT == QSR_OPT_ADAMW) p.s2[e] = b;
                 }
-                if (FUSE_MEAN) {
+                if (FUSE == FUSE_MEAN) {
                     const float mean = acc / float(p.K);
                     for (int k = 0; k < p.K; ++k) p.theta[int64_t(k) * p.stride + i] = mean;
+                } else if (FUSE == FUSE_SUM) {
+                    p.sum_out[i] = acc;
                 }
             }
         }
@@ -471,7 +479,7 @@ unsigned grid_for(int64_t P, int threads)
     return unsigned(blocks);
 }
 
-template <int OPT, bool EXT, bool FUSE>
+template <int OPT, bool EXT, int FUSE>
 int launch_step_rows(const StepParams &p, const LaunchShape &s, cudaStream_t st)
 {
     const unsigned grid = grid_for(p.P, s.step_threads);
@@ -485,7 +493,7 @@ int launch_step_rows(const StepParams &p, const LaunchShape &s, cudaStream_t st)
     return int(cudaGetLastError());
 }
 
-template <bool FUSE>
+template <int FUSE>
 int launch_step_any(const StepParams &p, int opt, const LaunchShape &shape, cudaStream_t st)
 {
     const bool ext = p.grads != nullptr;
@@ -500,12 +508,17 @@ int launch_step_any(const StepParams &p, int opt, const LaunchShape &shape, cuda
 
 int launch_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream)
 {
-    return launch_step_any<false>(p, opt, shape, static_cast<cudaStream_t>(stream));
+    return launch_step_any<FUSE_NONE>(p, opt, shape, static_cast<cudaStream_t>(stream));
 }
 
 int launch_step_mean(const StepParams &p, int opt, const LaunchShape &shape, void *stream)
 {
-    return launch_step_any<true>(p, opt, shape, static_cast<cudaStream_t>(stream));
+    return launch_step_any<FUSE_MEAN>(p, opt, shape, static_cast<cudaStream_t>(stream));
+}
+
+int launch_step_sum(const StepParams &p, int opt, const LaunchShape &shape, void *stream)
+{
+    return launch_step_any<FUSE_SUM>(p, opt, shape, static_cast<cudaStream_t>(stream));
 }
 
 int launch_parallel_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream)

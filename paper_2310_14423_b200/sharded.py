@@ -3,8 +3,9 @@
 This is the paper's own layout -- one worker (here: a block of workers) per GPU, parameters averaged by an
 All-Reduce at the end of each round -- and the only exchange step on the path: local steps need no
 communication.  Per round each process
-    1. takes H local steps on its rows                                  (qsr_local_step, H launches)
-    2. sums its rows' parameters into a [P] buffer                      (qsr_sync_partial)
+    1. takes H - 1 local steps on its rows                              (qsr_local_step)
+    2. takes the last step and sums its rows' new parameters into a [P] buffer, in one launch that does not even
+       write the parameter rows                                         (qsr_local_step_partial)
     3. all-reduces that buffer (SUM) over processes                     (torch.distributed: NCCL over NVLink)
     4. divides by the global worker count and writes every local row    (qsr_sync_finish)
 The round length comes from the host schedule, which depends only on t, so every process computes the same H
@@ -36,9 +37,9 @@ def run_rounds(engine, sums, K_total: int, t_begin: int, t_end: int, all_reduce)
     t = int(t_begin)
     while t < t_end:
         H = engine.qsr_round_length(t)
-        for h in range(H):
+        for h in range(H - 1):
             engine.qsr_local_step(t + h)
-        engine.qsr_sync_partial(sums)
+        engine.qsr_local_step_partial(t + H - 1, sums)    # last step + this process's row sums, one launch
         all_reduce(sums)
         engine.qsr_sync_finish(sums, K_total, t + H)
         rounds.append((t, H))

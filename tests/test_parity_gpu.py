@@ -244,11 +244,15 @@ def test_sharded_sync_equals_single_process():
         while t < w.T:
             H = parts[0][1].qsr_round_length(t)
             assert H == parts[1][1].qsr_round_length(t)
-            for h in range(H):
+            for h in range(H - 1):
                 for S, ctx in parts:
                     ctx.qsr_local_step(t + h)
-            for (S, ctx), buf in zip(parts, sums):
-                ctx.qsr_sync_partial(buf)
+            for r, ((S, ctx), buf) in enumerate(zip(parts, sums)):
+                if r == 0:                       # one rank takes the two-launch route, the other the fused one
+                    ctx.qsr_local_step(t + H - 1)
+                    ctx.qsr_sync_partial(buf)
+                else:
+                    ctx.qsr_local_step_partial(t + H - 1, buf)
             total = sums[0] + sums[1]
             for S, ctx in parts:
                 ctx.qsr_sync_finish(total, 6, t + H)

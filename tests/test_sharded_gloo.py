@@ -34,7 +34,8 @@ class OracleEngine:
     def qsr_local_step(self, t):
         self.S.local_step(t)
 
-    def qsr_sync_partial(self, sums):
+    def qsr_local_step_partial(self, t, sums):
+        self.S.local_step(t)
         sums.copy_(torch.from_numpy(self.S.theta.sum(axis=0)))
 
     def qsr_sync_finish(self, sums, K_total, t_next):
