@@ -1,8 +1,10 @@
 // C ABI of the library: argument checks, host-side scalars of each step, launches.  See include/qsr.h.
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <cmath>
 #include <cstdint>
+#include <cstdio>
 #include <cstring>
 #include <new>
 
@@ -76,6 +78,17 @@ qsr::SyncParams sync_params(const qsr_ctx &x)
 }
 
 int cuda_rc(int err) { return err == 0 ? QSR_OK : QSR_ECUDA; }
+
+// NVTX range for one communication round; a no-op unless a profiler is attached.
+struct RoundRange {
+    RoundRange(int64_t s, int64_t t, int64_t H)
+    {
+        char name[64];
+        std::snprintf(name, sizeof name, "qsr round %lld: t=%lld H=%lld", (long long)s, (long long)t, (long long)H);
+        nvtxRangePushA(name);
+    }
+    ~RoundRange() { nvtxRangePop(); }
+};
 
 // With clipping on: enqueue the norm pass and the factor pass for this step and make the step kernel use the factors.
 int prepare_clip(qsr_ctx &x, qsr::StepParams &p, bool parallel)
@@ -311,6 +324,7 @@ int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
     int64_t s = 0;
     for (int64_t t = t_begin; t < t_end;) {
         const int64_t H = qsr::round_length(ctx->cfg, t);       // GetH
+        const RoundRange range(s, t, H);
         for (int64_t h = 0; h + 1 < H; ++h)
             if (int rc = qsr_local_step(ctx, t + h, nullptr)) return rc;
         // the round's last step and the parameter averaging, in one launch when the state is kept per worker
