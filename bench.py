@@ -11,8 +11,9 @@ the timed window covers global steps [0, K) of its 10,000-step schedule.
 
 metric  replica param-updates per second = (workers x parameters x steps) / time, whole job, inputs resident in HBM.
 e2e     the same through qsr_train_host: host buffers in, host buffer out, copies inside the timed region.
-With N > 1 (torchrun, one rank per GPU) the workers are sharded over ranks (16 per GPU, weak scaling); each round's
-averaging is a partial-sum kernel, one NCCL all-reduce of P floats and a finish kernel.
+With N > 1 (torchrun, one rank per GPU) the workers are sharded over ranks (16 per GPU, weak scaling); a round ends
+with its last step fused with the rank's row sums, one NCCL all-reduce of P floats and a finish kernel.  On one GPU
+a round's last step carries the averaging itself (one launch, no extra HBM traffic).
 
 `--impl reference` times the CPU oracle (test infrastructure; plain C, binary64) on the host cores instead.
 """
@@ -43,8 +44,8 @@ FALLBACK_HBM_GBS = 6650.0
 # once, so traffic grows in proportion to K*P).  Valid only for the kernel source it was taken from: the hash covers
 # the noise generator, the optimizer update and local_step_kernel in csrc/kernels.cu.
 NCU_TRAFFIC = {
-    "step_source_sha256": "bf4023c4b1c52a79baf4977b409ea2f8f6fbf8b2f3bdf9a0bfdafcffbe5e8d66",
-    "bytes_per_update": {"adamw": 24.068, "sgdm": 16.069},
+    "step_source_sha256": "bf53f91172571ab3f60ce34230abce8d4f1f4a2636c499fc64e79fe05f4ba737",
+    "bytes_per_update": {"adamw": 24.083, "sgdm": 16.070},
 }
 
 
