@@ -44,8 +44,8 @@ FALLBACK_HBM_GBS = 6650.0
 # once, so traffic grows in proportion to K*P).  Valid only for the kernel source it was taken from: the hash covers
 # the noise generator, the optimizer update and local_step_kernel in csrc/kernels.cu.
 NCU_TRAFFIC = {
-    "step_source_sha256": "bf53f91172571ab3f60ce34230abce8d4f1f4a2636c499fc64e79fe05f4ba737",
-    "bytes_per_update": {"adamw": 24.083, "sgdm": 16.070},
+    "step_source_sha256": "9fa08dcb6994aef47cc62a683a71a87c749e3903f68660629afb8695d1638d86",
+    "bytes_per_update": {"adamw": 24.067, "sgdm": 16.073},
 }
 
 

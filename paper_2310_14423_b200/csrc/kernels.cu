@@ -126,14 +126,16 @@ __device__ __forceinline__ float4 div4(float4 x, float d) { return make_float4(x
 // reported by the launch as an error, not silently spilled.
 enum { FUSE_NONE = 0, FUSE_MEAN = 1, FUSE_SUM = 2 };
 
-template <int OPT, bool EXT_GRAD, int ROWS, int FUSE>
+// EXTRAS selects the build that honours the per-tensor weight-decay table and the clipping factors; the plain build
+// (no table, clipping off: every run of the paper's QSR experiments) does not carry their tests in the row loop.
+template <int OPT, bool EXT_GRAD, int ROWS, int FUSE, bool EXTRAS>
 __global__ void local_step_kernel(const StepParams p)
 {
     const int64_t n_col = (p.P + 3) >> 2;
     const int64_t grid_stride = int64_t(gridDim.x) * blockDim.x;
     for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < n_col; j += grid_stride) {
         const int64_t i0 = j << 2;
-        const float wdv = weight_decay_at<OPT>(p, i0);
+        const float wdv = EXTRAS ? weight_decay_at<OPT>(p, i0) : (OPT == QSR_OPT_SGDM ? p.wd : p.eta_wd);
         if (i0 + 4 <= p.P) {
             float4 lam = make_float4(0.f, 0.f, 0.f, 0.f), ths = lam;
             if (!EXT_GRAD) {
@@ -164,7 +166,7 @@ __global__ void local_step_kernel(const StepParams p)
                             g[r].z = fmaf(p.sigma, z.z, lam.z * (th[r].z - ths.z));
                             g[r].w = fmaf(p.sigma, z.w, lam.w * (th[r].w - ths.w));
                         }
-                        if (p.clip_coef) {   // gradient clipping: this worker's factor min(1, c / (||g|| + 1e-6))
+                        if (EXTRAS && p.clip_coef) {   // gradient clipping: this worker's factor min(1, c / (||g|| + 1e-6))
                             const float cs = __ldg(p.clip_coef + k + r);
                             g[r].x *= cs; g[r].y *= cs; g[r].z *= cs; g[r].w *= cs;
                         }
@@ -202,7 +204,7 @@ __global__ void local_step_kernel(const StepParams p)
                         const float zc = c == 0 ? z.x : (c == 1 ? z.y : z.z);
                         g = fmaf(p.sigma, zc, p.lambda[i] * (th - p.theta_star[i]));
                     }
-                    if (p.clip_coef) g *= __ldg(p.clip_coef + k);
+                    if (EXTRAS && p.clip_coef) g *= __ldg(p.clip_coef + k);
                     opt_update<OPT>(th, a, b, g, p, wdv);
                     if (FUSE != FUSE_NONE) acc += th;
                     else p.theta[e] = th;
@@ -484,11 +486,20 @@ int launch_step_rows(const StepParams &p, const LaunchShape &s, cudaStream_t st)
 {
     const unsigned grid = grid_for(p.P, s.step_threads);
     const int rows = s.step_rows ? s.step_rows : (OPT == QSR_OPT_ADAMW ? 4 : 2);
-    switch (rows) {
-    case 1: local_step_kernel<OPT, EXT, 1, FUSE><<<grid, s.step_threads, 0, st>>>(p); break;
-    case 2: local_step_kernel<OPT, EXT, 2, FUSE><<<grid, s.step_threads, 0, st>>>(p); break;
-    case 4: local_step_kernel<OPT, EXT, 4, FUSE><<<grid, s.step_threads, 0, st>>>(p); break;
-    default: local_step_kernel<OPT, EXT, 8, FUSE><<<grid, s.step_threads, 0, st>>>(p); break;
+    if (p.n_tensors > 0 || p.clip_coef) {
+        switch (rows) {
+        case 1: local_step_kernel<OPT, EXT, 1, FUSE, true><<<grid, s.step_threads, 0, st>>>(p); break;
+        case 2: local_step_kernel<OPT, EXT, 2, FUSE, true><<<grid, s.step_threads, 0, st>>>(p); break;
+        case 4: local_step_kernel<OPT, EXT, 4, FUSE, true><<<grid, s.step_threads, 0, st>>>(p); break;
+        default: local_step_kernel<OPT, EXT, 8, FUSE, true><<<grid, s.step_threads, 0, st>>>(p); break;
+        }
+    } else {
+        switch (rows) {
+        case 1: local_step_kernel<OPT, EXT, 1, FUSE, false><<<grid, s.step_threads, 0, st>>>(p); break;
+        case 2: local_step_kernel<OPT, EXT, 2, FUSE, false><<<grid, s.step_threads, 0, st>>>(p); break;
+        case 4: local_step_kernel<OPT, EXT, 4, FUSE, false><<<grid, s.step_threads, 0, st>>>(p); break;
+        default: local_step_kernel<OPT, EXT, 8, FUSE, false><<<grid, s.step_threads, 0, st>>>(p); break;
+        }
     }
     return int(cudaGetLastError());
 }
