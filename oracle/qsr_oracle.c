@@ -20,6 +20,10 @@
  *                     L2 weight decay (App. C.1) or AdamW with decoupled weight decay (App. C.2).
  *   orc_sync          the All-Reduce line of Algorithm 2: the next global iterate is the mean of
  *                     the workers' local iterates, which every worker then copies.
+ *   orc_parallel_step Algorithm 1 (Parallel OPT): the K gradients are taken at one point, averaged (the
+ *                     All-Reduce line) and fed to one OPT step.
+ *   gradient clipping inside orc_local_step: each worker's gradient scaled by min(1, c/(||g|| + 1e-6))
+ *                     before OPT (App. C.2; the form is that of the paper's software).
  *   orc_run           Algorithm 2 as a whole: rounds of GetH, local steps, averaging, t += H.
  *   orc_philox4x32_10 the Philox-4x32-10 counter-based generator (Salmon, Moraes, Dror, Shaw,
  *                     "Parallel random numbers: as easy as 1, 2, 3", SC'11), and orc_noise, the
@@ -34,10 +38,14 @@
  * prints in Tables 1-3 and against threshold crossings derived by inverting the cosine; SGD against
  * the closed-form solution of the heavy-ball recurrence and against torch.optim.SGD; AdamW against
  * torch.optim.AdamW and the constant-gradient closed form; the mean against its invariants; Philox
- * against the known-answer vectors published with the generator; the normal against its moments.
+ * against the known-answer vectors published with the generator; the normal against its moments;
+ * the other rules and schedules against the 13.2 % / 14.4 % of App. G's step-decay table and against
+ * threshold crossings; Algorithm 1 against torch.optim with the mean gradient and the H = 1 remark of
+ * Sec. 3; clipping against torch's clip_grad_norm_; per-tensor weight decay against torch parameter groups.
  * Parity unpinned by the paper (a stated reading only): the round length used during warm-up when
  * (alpha/eta_max)^2 exceeds H_base, the warm-up's first value (eta_0 = 0), what happens to
- * optimizer state at a synchronization (kept per worker), and uniform weight decay on all tensors.
+ * optimizer state at a synchronization (kept per worker), uniform weight decay on all tensors, and the
+ * exact round boundaries of the post-local and modified-SWAP schedules (the paper prints no number for them).
  */
 #include <math.h>
 #include <stdint.h>

@@ -219,12 +219,12 @@ int qsr_parallel_step(qsr_ctx *ctx, int64_t t, const float *grads)
 int qsr_local_step_sync(qsr_ctx *ctx, int64_t t, const float *grads, int64_t t_next)
 {
     if (!ctx) return QSR_EINVAL;
+    if (t < 0 || t >= ctx->cfg.T || t < ctx->t_state_origin || t_next < 0 || t_next > ctx->cfg.T) return QSR_ERANGE;
     if (ctx->cfg.state_sync != QSR_STATE_KEEP) {
         // Averaging or resetting the optimizer state needs the stand-alone kernel: two launches.
         if (int rc = qsr_local_step(ctx, t, grads)) return rc;
         return qsr_sync(ctx, t_next);
     }
-    if (t < 0 || t >= ctx->cfg.T || t < ctx->t_state_origin || t_next < 0 || t_next > ctx->cfg.T) return QSR_ERANGE;
     if (!grads && !ctx->lambda) return QSR_EINVAL;
     if (!aligned16(grads)) return QSR_EALIGN;
     qsr::StepParams p = step_params(*ctx, t, grads);

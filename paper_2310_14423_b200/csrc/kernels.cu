@@ -310,13 +310,6 @@ __global__ void parallel_step_kernel(const StepParams p)
 
 // ---------------------------------------------------------------------------------------------- gradient clipping
 
-// Pass 1 of global-norm clipping (App. C.2): partial sums of g^2, per worker (PARALLEL = false: one sum per row k of
-// the gradient that worker's step will use) or of the averaged gradient (PARALLEL = true: Algorithm 1).  Generated
-// gradients are recomputed here with the very expressions of the step kernel -- the noise is a pure function of
-// (seed, worker, step, coordinate) -- so nothing has to be stored: the pass reads theta once (4 B per update).
-// The grid is fixed (kNormGrid blocks at most) so that the partials fit a small workspace; a thread strides over
-// columns and keeps its running sum for worker k in shared memory at acc[k * blockDim.x + threadIdx.x].
-// partial is [gridDim.x, rows] with rows = PARALLEL ? 1 : K.  Summation order is fixed: results are deterministic.
 // 16-byte load when the whole column lies inside the row, scalar loads (zeros beyond P) for the ragged last column.
 __device__ __forceinline__ float4 ld4_guarded(const float *q, int valid)
 {
@@ -324,6 +317,13 @@ __device__ __forceinline__ float4 ld4_guarded(const float *q, int valid)
     return make_float4(q[0], valid > 1 ? q[1] : 0.f, valid > 2 ? q[2] : 0.f, 0.f);
 }
 
+// Pass 1 of global-norm clipping (App. C.2): partial sums of g^2, per worker (PARALLEL = false: one sum per row k of
+// the gradient that worker's step will use) or of the averaged gradient (PARALLEL = true: Algorithm 1).  Generated
+// gradients are recomputed here with the very expressions of the step kernel -- the noise is a pure function of
+// (seed, worker, step, coordinate) -- so nothing has to be stored: the pass reads theta once (4 B per update).
+// The grid is fixed (kNormGrid blocks at most) so that the partials fit a small workspace; a thread strides over
+// columns and keeps its running sum for worker k in shared memory at acc[k * blockDim.x + threadIdx.x].
+// partial is [gridDim.x, rows] with rows = PARALLEL ? 1 : K.  Summation order is fixed: results are deterministic.
 template <bool EXT_GRAD, bool PARALLEL>
 __global__ void grad_sqnorm_kernel(const StepParams p, float *partial)
 {
