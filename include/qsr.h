@@ -225,9 +225,10 @@ int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
 /* Kernel launches issued through this context so far. */
 int64_t qsr_launch_count(const qsr_ctx *ctx);
 
-/* Overrides the launch shape of the step kernel (threads per block: 64..1024, a multiple of 32; rows in flight
- * per thread: 1, 2, 4 or 8) and of the sync kernel (threads per block: 64..512).  0 keeps the current value.  A
- * step shape whose registers do not fit on an SM makes the next qsr_local_step return QSR_ECUDA. */
+/* Overrides the launch shape of the step kernel (threads per block: 64..1024, a multiple of 32; rows in flight per
+ * thread, i.e. the depth of its cp.async ring: 1, 2, 4 or 8) and of the sync kernel (threads per block: 64..512).
+ * 0 keeps the current value.  The ring takes rows x operands x threads x 16 bytes of shared memory (operands: 2 for
+ * SGD, 3 for AdamW, one more with a gradient slab); a shape beyond 227 KB makes the next step return QSR_ECUDA. */
 int qsr_set_launch_shape(qsr_ctx *ctx, int32_t step_threads, int32_t step_rows_in_flight, int32_t sync_threads);
 
 /* ---- whole run from host memory ----------------------------------------------------------------------- */

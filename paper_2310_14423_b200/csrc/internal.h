@@ -51,11 +51,11 @@ struct SyncParams {
 };
 
 struct LaunchShape {
-    // Defaults from sustained sweeps on B200 at the ViT-B/16 and ResNet-152 shapes (K = 16): 128-thread blocks; rows
-    // in flight per thread 4 for AdamW (three slabs to cover), 2 for SGD.  Grids capped at a few CTAs per SM with a
-    // grid-stride loop were 15-30 % slower than one CTA per 128 columns.
-    int step_threads = 128;
-    int step_rows = 0;        // 0 = pick by optimizer
+    // Defaults from sustained sweeps on B200 at the ViT-B/16 and ResNet-152 shapes (K = 16): 256-thread blocks with
+    // an 8-row cp.async ring per thread.  Grids capped at a few CTAs per SM with a grid-stride loop were 15-30 %
+    // slower than one thread per column.
+    int step_threads = 256;
+    int step_rows = 0;        // rows in flight per thread (ring depth); 0 = default (8)
     int sync_threads = 128;
 };
 
