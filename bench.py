@@ -38,14 +38,15 @@ METRIC = "replica_param_updates_per_s"
 UNIT = "param-updates/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+L2_BYTES = 126e6
 
 # DRAM traffic of the dominant kernel from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum per launch,
 # taken on the 2^23-parameter variants c4s / c3s and stated per element-update: the kernel streams every element
 # once, so traffic grows in proportion to K*P).  Valid only for the kernel source it was taken from: the hash covers
 # the noise generator, the optimizer update and local_step_kernel in csrc/kernels.cu.
 NCU_TRAFFIC = {
-    "step_source_sha256": "9fa08dcb6994aef47cc62a683a71a87c749e3903f68660629afb8695d1638d86",
-    "bytes_per_update": {"adamw": 24.067, "sgdm": 16.073},
+    "step_source_sha256": "4cf7d4f54bb12ac0ca3a2255b7cd2c61671f4d2ae9a60de5cb55b949a7b2d16e",
+    "bytes_per_update": {"adamw": 24.066, "sgdm": 16.068},
 }
 
 
@@ -418,6 +419,10 @@ def main():
                                         "frac_of_measured": end_gbs / peak,
                                         "note": "last step fused with row sums + NCCL all-reduce of P floats + finish kernel"}
 
+    slab_bytes = (3 if w.opt == W.OPT_ADAMW else 2) * K_local * P4 * 4
+    l2_note = ("inputs larger than L2 (every launch streams the whole slabs)" if slab_bytes > 2 * L2_BYTES else
+               f"slabs of {slab_bytes / 2**20:.0f} MiB stay resident in the 126 MB L2 between launches and no flush is "
+               "done: a launch-bound small case, no HBM roofline claim")
     label = {"c4": "c4: ViT-B/16-shaped parameter set, Local AdamW + QSR",
              "c3": "c3: ResNet-152-shaped parameter set, Local SGD + QSR"}.get(w.name, w.name)
     out = {
@@ -426,7 +431,7 @@ def main():
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": label, "K_per_gpu": K_local, "K_total": K_total, "P": w.P, "opt": w.opt, "T": w.T,
                    "window": f"global steps [0,{steps}) of the schedule", "syncs_in_window": n_syncs,
-                   "l2": "inputs larger than L2 (every launch streams the whole slabs)",
+                   "l2": l2_note,
                    "parallelism": f"replica-sharded dp{world}" if sharded_path else "1 GPU, replicas as slab rows"},
         "roofline": roofline, "kernels": kernels, "gpu_launches": int(launches), "clocks": clocks,
     }
