@@ -45,7 +45,11 @@ qsr::StepParams step_params(const qsr_ctx &x, int64_t t, const float *grads)
     p.grads = grads; p.lambda = x.lambda; p.theta_star = x.theta_star;
     p.P = c.P; p.stride = c.row_stride; p.K = c.K;
     p.worker0 = uint32_t(c.worker_offset);
-    p.key0 = uint32_t(c.seed); p.key1 = uint32_t(c.seed >> 32);
+    // Philox-4x32 key schedule (Salmon et al., SC'11): the key halves advance by the Weyl constants every round
+    for (uint32_t r = 0; r < 10; ++r) {
+        p.round_key[2 * r] = uint32_t(c.seed) + r * 0x9E3779B9u;
+        p.round_key[2 * r + 1] = uint32_t(c.seed >> 32) + r * 0xBB67AE85u;
+    }
     p.step = uint32_t(t);
     p.sigma = float(c.noise_std);
     const double eta = qsr::learning_rate(c, t);

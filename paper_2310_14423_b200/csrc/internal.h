@@ -21,7 +21,7 @@ struct StepParams {
     int64_t P, stride;
     int32_t K;
     uint32_t worker0;         // global index of row 0
-    uint32_t key0, key1;      // Philox key (seed halves)
+    uint32_t round_key[20];   // Philox key schedule: round r uses (key0 + r*W0, key1 + r*W1) at [2r], [2r+1]
     uint32_t step;            // global iteration t (Philox counter word 2)
     float sigma;              // noise_std
     float eta, wd, mu;        // SGD with momentum

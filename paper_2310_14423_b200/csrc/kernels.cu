@@ -17,17 +17,17 @@ namespace {
 
 // ---------------------------------------------------------------------------------------------- noise
 
-// Philox-4x32 with 10 rounds (Salmon et al., SC'11): 128-bit counter, 64-bit key.
-__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1)
+// Philox-4x32 with 10 rounds (Salmon et al., SC'11): 128-bit counter, 64-bit key.  The key schedule
+// (key + r * Weyl constant) does not depend on the counter, so the host evaluates it once per launch and the ten
+// round keys arrive as kernel arguments: a round is two 32x32->64 multiplies and two three-input XORs.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, const uint32_t (&rk)[20])
 {
-    constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
-        const uint32_t hi0 = __umulhi(M0, c.x), lo0 = M0 * c.x;
-        const uint32_t hi1 = __umulhi(M1, c.z), lo1 = M1 * c.z;
-        c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
-        k0 += W0;
-        k1 += W1;
+        const uint64_t p0 = uint64_t(M0) * c.x, p1 = uint64_t(M1) * c.z;
+        c = make_uint4(uint32_t(p1 >> 32) ^ c.y ^ rk[2 * r], uint32_t(p1), uint32_t(p0 >> 32) ^ c.w ^ rk[2 * r + 1],
+                       uint32_t(p0));
     }
     return c;
 }
@@ -42,28 +42,78 @@ __device__ __forceinline__ float sqrt_fast(float x)
     return y;
 }
 
+// -2 ln(u) for u = (a + 1/2) / 2^23, a = the top 23 bits of w: u is exact in fp32 and lies in [2^-24, 1 - 2^-24].
+// The 23 bits are dropped into the mantissa of a float in [1, 2) and shifted down by an exact subtraction (no
+// integer-to-float conversion).  ln(u) = e ln 2 + ln(m) with u = m 2^e, m in [2/3, 4/3); ln(m) = f + f^2 Q(f), f = m - 1,
+// Q a degree-7 minimax fit of (ln(1+f) - f) / f^2 on [-1/3, 1/3] (|error| < 1.7e-7, i.e. < 6e-8 relative to ln m).
+// The input range is known, so none of a general logf's tests for zero, negative, infinite or subnormal arguments is
+// needed.  Over all 2^23 values of a the relative error of the result is below 1.0e-7 with no bias in the mean.
+__device__ __forceinline__ float neg2_log_unit(uint32_t w)
+{
+    const float u = __uint_as_float(0x3f800000u | (w >> 9)) - (1.0f - 0x1p-24f);      // (a + 1/2) / 2^23, exact
+    const int t = __float_as_int(u) - 0x3f2aaaab;                                     // 0x3f2aaaab: bits of 2/3
+    const float m = __int_as_float((t & 0x007fffff) + 0x3f2aaaab);
+    const float e = __int_as_float(0x4b400000 + (t >> 23)) - 12582912.0f;             // exponent as a float, exact
+    const float f = m - 1.0f;
+    float q = 0.14067277312278748f;
+    q = fmaf(q, f, -0.15009641647338867f);
+    q = fmaf(q, f, 0.13995099067687988f);
+    q = fmaf(q, f, -0.16489295661449432f);
+    q = fmaf(q, f, 0.20010477304458618f);
+    q = fmaf(q, f, -0.2500377893447876f);
+    q = fmaf(q, f, 0.3333323299884796f);
+    q = fmaf(q, f, -0.49999991059303284f);
+    const float ln_m = fmaf(f * f, q, f);
+    return -2.0f * fmaf(e, 0.6931471805599453f, ln_m);
+}
+
+// cos and sin of the angle 2 pi (b + 1/2) / 2^23, b = the top 23 bits of w.  In quarter turns the angle is
+// x = (b + 1/2) / 2^21 = n + y with n = round(x) and y in (-1/2, 1/2); n mod 4 is the top two bits of
+// w + 2^29 (the addition wraps at a full turn), the next 21 bits are y + 1/2 up to the half-unit offset, and they
+// become a float by the same mantissa trick, so the argument reduction is exact and costs four integer/float
+// instructions.  sin(pi/2 y) and cos(pi/2 y) are degree-7 / degree-8 minimax polynomials (|error| < 3e-9 / 2e-10);
+// the quadrant swaps them and sets the signs with the same top bits.  Over all 2^23 angles: |error| < 9e-8, mean 0.
+__device__ __forceinline__ void sincos_turn_bits(uint32_t w, float &sin_out, float &cos_out)
+{
+    const uint32_t t = w + 0x20000000u;
+    const float y = __uint_as_float(((t >> 7) & 0x007ffffcu) | 0x3f800000u) - (1.5f - 0x1p-22f);
+    const float y2 = y * y;
+    float ps = -0.004602177068591118f;
+    ps = fmaf(ps, y2, 0.07968022674322128f);
+    ps = fmaf(ps, y2, -0.6459634900093079f);
+    ps = fmaf(ps, y2, 1.5707963705062866f);
+    const float s = y * ps;
+    float pc = 0.0009067608625628054f;
+    pc = fmaf(pc, y2, -0.020861538127064705f);
+    pc = fmaf(pc, y2, 0.253669410943985f);
+    pc = fmaf(pc, y2, -1.2337005138397217f);
+    const float c = fmaf(pc, y2, 1.0f);
+    const bool odd = (t & 0x40000000u) != 0;                  // n odd: sine and cosine trade places
+    const float c0 = odd ? s : c, s0 = odd ? c : s;
+    // signs: sin < 0 for n in {2, 3} (bit 31 of t), cos < 0 for n in {1, 2} (bit 31 of t + 2^30)
+    sin_out = __uint_as_float(__float_as_uint(s0) ^ (t & 0x80000000u));
+    cos_out = __uint_as_float(__float_as_uint(c0) ^ ((t + 0x40000000u) & 0x80000000u));
+}
+
 // Box-Muller on two words: uniforms are (top 23 bits + 1/2) / 2^23, exact in fp32 and never 0 or 1.
-// The 23 bits are dropped into the mantissa of a float in [1, 2) and shifted down by an exact subtraction, which keeps
-// the integer-to-float conversions off the special-function pipe.  log and sincospi stay the accurate library
-// versions: their errors are unbiased (measured mean error of sincospif on the 2^23-point grid: < 1e-16), and a bias
-// of 1e-8 in the noise would move the fixed point of a coordinate with curvature 1e-3 by 1e-5 * sigma.
+// Both transcendental parts are written for exactly these inputs (see above) rather than taken from the math library:
+// the generic logf and sincospif cost about twice the instructions, and the step kernel is bound by instruction issue
+// almost as much as by memory.  Their errors stay rounding-sized and unbiased; a bias of 1e-8 in the noise would move
+// the fixed point of a coordinate with curvature 1e-3 by 1e-5 * sigma, which is why the hardware's approximate
+// sine/cosine (biased by about -1.3e-8 on this grid) is not used.
 __device__ __forceinline__ void box_muller(uint32_t wa, uint32_t wb, float &z_cos, float &z_sin)
 {
-    const float fa = __uint_as_float(0x3f800000u | (wa >> 9));    // 1 + a / 2^23
-    const float fb = __uint_as_float(0x3f800000u | (wb >> 9));
-    const float u1 = fa - (1.0f - 0x1p-24f);                      // (a + 1/2) / 2^23, exact
-    const float two_u2 = fmaf(2.0f, fb, -(2.0f - 0x1p-23f));      // (b + 1/2) / 2^22 = angle / pi, exact
-    const float radius = sqrt_fast(-2.0f * logf(u1));
+    const float radius = sqrt_fast(neg2_log_unit(wa));
     float s, c;
-    sincospif(two_u2, &s, &c);
+    sincos_turn_bits(wb, s, c);
     z_cos = radius * c;
     z_sin = radius * s;
 }
 
 // Four standard normals for coordinates 4j .. 4j+3 of one worker at one step.
-__device__ __forceinline__ float4 noise4(int64_t j, uint32_t step, uint32_t worker, uint32_t key0, uint32_t key1)
+__device__ __forceinline__ float4 noise4(int64_t j, uint32_t step, uint32_t worker, const uint32_t (&rk)[20])
 {
-    const uint4 r = philox4x32_10(make_uint4(uint32_t(j), uint32_t(uint64_t(j) >> 32), step, worker), key0, key1);
+    const uint4 r = philox4x32_10(make_uint4(uint32_t(j), uint32_t(uint64_t(j) >> 32), step, worker), rk);
     float4 z;
     box_muller(r.x, r.y, z.x, z.y);
     box_muller(r.z, r.w, z.z, z.w);
@@ -157,7 +207,7 @@ struct StepOperands {
 };
 
 template <int OPT, bool EXT_GRAD, int STAGES, int FUSE, bool EXTRAS>
-__global__ void local_step_kernel(const StepParams p)
+__global__ void local_step_kernel(const __grid_constant__ StepParams p)
 {
     extern __shared__ float4 ring[];   // [STAGES][operands][blockDim.x]
     constexpr int NOP = StepOperands<OPT, EXT_GRAD>::kCount;
@@ -199,7 +249,7 @@ __global__ void local_step_kernel(const StepParams p)
                 cp_async_commit();
                 stage = stage + 1 == STAGES ? 0 : stage + 1;
                 if (!EXT_GRAD) {
-                    const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.key0, p.key1);
+                    const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.round_key);
                     g.x = fmaf(p.sigma, z.x, lam.x * (th.x - ths.x));
                     g.y = fmaf(p.sigma, z.y, lam.y * (th.y - ths.y));
                     g.z = fmaf(p.sigma, z.z, lam.z * (th.z - ths.z));
@@ -238,7 +288,7 @@ __global__ void local_step_kernel(const StepParams p)
                     if (EXT_GRAD) {
                         g = p.grads[e];
                     } else {
-                        const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.key0, p.key1);
+                        const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.round_key);
                         const float zc = c == 0 ? z.x : (c == 1 ? z.y : z.z);
                         g = fmaf(p.sigma, zc, p.lambda[i] * (th - p.theta_star[i]));
                     }
@@ -283,7 +333,7 @@ __device__ __forceinline__ float4 column_sum(const float *slab, int64_t i0, int6
 // HBM traffic is that of one row (plus the K gradient rows when they come from a slab); with generated gradients the
 // kernel is bound by the K noise evaluations per coordinate, not by memory.
 template <int OPT, bool EXT_GRAD>
-__global__ void parallel_step_kernel(const StepParams p)
+__global__ void parallel_step_kernel(const __grid_constant__ StepParams p)
 {
     const int64_t n_col = (p.P + 3) >> 2;
     const int64_t grid_stride = int64_t(gridDim.x) * blockDim.x;
@@ -302,7 +352,7 @@ __global__ void parallel_step_kernel(const StepParams p)
                 const float4 pull = make_float4(lam.x * (th.x - ths.x), lam.y * (th.y - ths.y),
                                                 lam.z * (th.z - ths.z), lam.w * (th.w - ths.w));
                 for (int k = 0; k < p.K; ++k) {
-                    const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.key0, p.key1);
+                    const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.round_key);
                     sum.x += fmaf(p.sigma, z.x, pull.x);
                     sum.y += fmaf(p.sigma, z.y, pull.y);
                     sum.z += fmaf(p.sigma, z.z, pull.z);
@@ -330,7 +380,7 @@ __global__ void parallel_step_kernel(const StepParams p)
                     if (EXT_GRAD) {
                         sum += p.grads[int64_t(k) * p.stride + i];
                     } else {
-                        const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.key0, p.key1);
+                        const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.round_key);
                         const float zc = c == 0 ? z.x : (c == 1 ? z.y : z.z);
                         sum += fmaf(p.sigma, zc, p.lambda[i] * (th - p.theta_star[i]));
                     }
@@ -363,7 +413,7 @@ __device__ __forceinline__ float4 ld4_guarded(const float *q, int valid)
 // columns and keeps its running sum for worker k in shared memory at acc[k * blockDim.x + threadIdx.x].
 // partial is [gridDim.x, rows] with rows = PARALLEL ? 1 : K.  Summation order is fixed: results are deterministic.
 template <bool EXT_GRAD, bool PARALLEL>
-__global__ void grad_sqnorm_kernel(const StepParams p, float *partial)
+__global__ void grad_sqnorm_kernel(const __grid_constant__ StepParams p, float *partial)
 {
     extern __shared__ float acc[];
     const int rows = PARALLEL ? 1 : p.K;
@@ -386,7 +436,7 @@ __global__ void grad_sqnorm_kernel(const StepParams p, float *partial)
             } else {
                 // Algorithm 1 evaluates every worker's gradient at the single model in row 0
                 const float4 th = ld4_guarded(p.theta + int64_t(PARALLEL ? 0 : k) * p.stride + i0, valid);
-                const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.key0, p.key1);
+                const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.round_key);
                 g.x = fmaf(p.sigma, z.x, lam.x * (th.x - ths.x));
                 g.y = valid > 1 ? fmaf(p.sigma, z.y, lam.y * (th.y - ths.y)) : 0.f;
                 g.z = valid > 2 ? fmaf(p.sigma, z.z, lam.z * (th.z - ths.z)) : 0.f;
