@@ -45,8 +45,8 @@ L2_BYTES = 126e6
 # once, so traffic grows in proportion to K*P).  Valid only for the kernel source it was taken from: the hash covers
 # the noise generator, the optimizer update and local_step_kernel in csrc/kernels.cu.
 NCU_TRAFFIC = {
-    "step_source_sha256": "4cf7d4f54bb12ac0ca3a2255b7cd2c61671f4d2ae9a60de5cb55b949a7b2d16e",
-    "bytes_per_update": {"adamw": 24.066, "sgdm": 16.068},
+    "step_source_sha256": "ff2976835143924ba17aaf60339c53736ec7b83cadb9db352fc744aec8fd6278",
+    "bytes_per_update": {"adamw": 24.064, "sgdm": 16.069},
 }
 
 

@@ -222,7 +222,20 @@ int qsr_sync_static(qsr_ctx *ctx, int64_t t_next);
 int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
             int64_t *round_start, int64_t *round_len, int64_t cap, int64_t *n_rounds);
 
-/* Kernel launches issued through this context so far. */
+/* Replays qsr_run's launches from CUDA graphs (Algorithm 2's round as one graph).  For small parameter sets a local
+ * step takes a few microseconds on the device and a run is bound by the cost of launching H(s) kernels per round;
+ * with max_steps_per_graph = G > 0, qsr_run enqueues each round as chains of at most G step kernels, each chain one
+ * graph launch (a round's last chain ends in the fused step-and-average launch when state_sync = QSR_STATE_KEEP).
+ * A chain of a given length is built and instantiated once, kept in the context (at most 48 distinct lengths; beyond
+ * that, and whenever gradient clipping is on, qsr_run launches directly as before) and replayed with the arguments of
+ * its steps -- learning rate, bias corrections, noise counter -- rewritten on the host before every replay.  The
+ * kernels, their order and their arguments are those of the direct path, so the results are bit-identical.
+ * G = 0 (the default) switches replay off.  QSR_ERANGE unless 0 <= G <= 1024.  qsr_train_host switches it on with
+ * G = 64 when one step moves at most 32 MiB.  Changing the launch shape discards the cached graphs.  qsr_run must
+ * not itself be called while its stream is being captured when replay is on. */
+int qsr_set_graph_replay(qsr_ctx *ctx, int32_t max_steps_per_graph);
+
+/* Kernel launches issued through this context so far (a replayed graph counts its kernels). */
 int64_t qsr_launch_count(const qsr_ctx *ctx);
 
 /* Overrides the launch shape of the step kernel (threads per block: 64..1024, a multiple of 32; rows in flight per

@@ -7,8 +7,20 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "internal.h"
+
+// A chain of step-kernel nodes that has been instantiated once and is replayed with new arguments: `n_plain` plain
+// steps, then (if `fused`) the round's last step with the replica mean.
+struct StepGraph {
+    int n_plain;
+    bool fused;
+    cudaGraph_t graph;
+    cudaGraphExec_t exec;
+    std::vector<cudaGraphNode_t> nodes;
+    qsr::StepLaunch plain, last;      // kernel instance and geometry of the plain nodes and of the fused last node
+};
 
 struct qsr_ctx {
     qsr_config cfg;
@@ -24,6 +36,8 @@ struct qsr_ctx {
     const float *wd_scale;
     double clip_norm;         // > 0: gradient clipping on
     float *clip_ws;           // caller's workspace for the norm partials and the factors
+    int32_t graph_steps;      // > 0: qsr_run replays its launches from CUDA graphs of at most this many steps
+    std::vector<StepGraph> graphs;
 };
 
 namespace {
@@ -99,10 +113,92 @@ int prepare_clip(qsr_ctx &x, qsr::StepParams &p, bool parallel)
 {
     if (!(x.clip_norm > 0.0)) return QSR_OK;
     const int rows = parallel ? 1 : x.cfg.K;
-    const int grid = qsr::clip_grid(x.cfg.P, x.shape.step_threads);
+    const int grid = qsr::clip_grid(x.cfg.P);
     x.launches += 2;
     if (int err = qsr::launch_clip_coef(p, parallel, x.clip_norm, x.clip_ws, x.shape, x.stream)) return cuda_rc(err);
     p.clip_coef = x.clip_ws + int64_t(grid) * rows;
+    return QSR_OK;
+}
+
+constexpr size_t kMaxCachedGraphs = 48;
+
+void drop_graphs(qsr_ctx &x)
+{
+    for (StepGraph &g : x.graphs) {
+        if (g.exec) cudaGraphExecDestroy(g.exec);
+        if (g.graph) cudaGraphDestroy(g.graph);
+    }
+    x.graphs.clear();
+}
+
+// Graph replay covers the launches qsr_run issues by itself: plain steps with generated gradients, and the fused
+// last step when the state is kept per worker.  Clipping adds two launches per step whose arguments move with the
+// workspace, so it stays on the direct path.
+bool graph_replay_applies(const qsr_ctx &x) { return x.graph_steps > 0 && !(x.clip_norm > 0.0); }
+
+cudaKernelNodeParams node_params(const qsr::StepLaunch &L, void **args)
+{
+    cudaKernelNodeParams k;
+    std::memset(&k, 0, sizeof k);
+    k.func = const_cast<void *>(L.func);
+    k.gridDim = dim3(L.grid);
+    k.blockDim = dim3(unsigned(L.threads));
+    k.sharedMemBytes = unsigned(L.smem);
+    k.kernelParams = args;
+    k.extra = nullptr;
+    return k;
+}
+
+// Steps t .. t + n_plain - 1 as plain local steps and, if `fused`, step t + n_plain as the round's last step with
+// the replica mean, enqueued as ONE graph launch.  The chain for (n_plain, fused) is built and instantiated the first
+// time it is needed and kept; every replay first rewrites each node's StepParams (the learning rate, the bias
+// corrections and the Philox counter word change with t).  An update only affects launches made after it, so the
+// executable graph may still be running an earlier replay while it is being updated.  Returns QSR_OK, QSR_ECUDA,
+// or 1 when the cache is full and the caller should launch directly.
+int replay_steps(qsr_ctx &x, int64_t t, int n_plain, bool fused)
+{
+    const int n = n_plain + (fused ? 1 : 0);
+    StepGraph *g = nullptr;
+    for (StepGraph &c : x.graphs)
+        if (c.n_plain == n_plain && c.fused == fused) { g = &c; break; }
+    std::vector<qsr::StepParams> params;
+    params.resize(size_t(n));
+    for (int i = 0; i < n; ++i) params[size_t(i)] = step_params(x, t + i, nullptr);
+    if (!g) {
+        if (x.graphs.size() >= kMaxCachedGraphs) return 1;
+        StepGraph fresh;
+        fresh.n_plain = n_plain; fresh.fused = fused; fresh.graph = nullptr; fresh.exec = nullptr;
+        if (qsr::resolve_step(params[0], x.cfg.opt, x.shape, qsr::FUSE_NONE, &fresh.plain) != 0 ||
+            qsr::resolve_step(params[0], x.cfg.opt, x.shape, qsr::FUSE_MEAN, &fresh.last) != 0)
+            return QSR_ECUDA;
+        if (cudaGraphCreate(&fresh.graph, 0) != cudaSuccess) return QSR_ECUDA;
+        bool ok = true;
+        for (int i = 0; i < n && ok; ++i) {
+            void *args[] = {&params[size_t(i)]};
+            const cudaKernelNodeParams k = node_params((fused && i == n - 1) ? fresh.last : fresh.plain, args);
+            cudaGraphNode_t node = nullptr;
+            const cudaGraphNode_t *dep = fresh.nodes.empty() ? nullptr : &fresh.nodes.back();
+            ok = cudaGraphAddKernelNode(&node, fresh.graph, dep, dep ? 1 : 0, &k) == cudaSuccess;
+            if (ok) fresh.nodes.push_back(node);
+        }
+        if (ok) ok = cudaGraphInstantiate(&fresh.exec, fresh.graph, 0) == cudaSuccess;
+        if (!ok) {
+            if (fresh.exec) cudaGraphExecDestroy(fresh.exec);
+            cudaGraphDestroy(fresh.graph);
+            cudaGetLastError();
+            return QSR_ECUDA;
+        }
+        x.graphs.push_back(fresh);
+        g = &x.graphs.back();     // instantiated with this replay's arguments: no update needed
+    } else {
+        for (int i = 0; i < n; ++i) {
+            void *args[] = {&params[size_t(i)]};
+            const cudaKernelNodeParams k = node_params((fused && i == n - 1) ? g->last : g->plain, args);
+            if (cudaGraphExecKernelNodeSetParams(g->exec, g->nodes[size_t(i)], &k) != cudaSuccess) return QSR_ECUDA;
+        }
+    }
+    if (cudaGraphLaunch(g->exec, x.stream) != cudaSuccess) return QSR_ECUDA;
+    x.launches += n;
     return QSR_OK;
 }
 
@@ -131,17 +227,20 @@ int qsr_init(qsr_ctx **out, const qsr_config *cfg, float *params, float *state1,
     x->lambda = lambda; x->theta_star = theta_star;
     x->stream = static_cast<cudaStream_t>(cuda_stream);
     x->shape = qsr::LaunchShape();
+    if (cfg->opt == QSR_OPT_SGDM) x->shape.step_threads = 128;
     x->t_state_origin = cfg->t_state_origin;
     x->launches = 0;
     x->partial_pending = false;
     x->n_tensors = 0; x->tensor_end = nullptr; x->wd_scale = nullptr;
     x->clip_norm = 0.0; x->clip_ws = nullptr;
+    x->graph_steps = 0;
     *out = x;
     return QSR_OK;
 }
 
 int qsr_destroy(qsr_ctx *ctx)
 {
+    if (ctx) drop_graphs(*ctx);
     delete ctx;
     return QSR_OK;
 }
@@ -203,7 +302,7 @@ int qsr_set_grad_clip(qsr_ctx *ctx, double max_norm, float *workspace_dev)
     }
     if (!workspace_dev) return QSR_EINVAL;
     if (!aligned16(workspace_dev)) return QSR_EALIGN;
-    if (ctx->cfg.K > 96) return QSR_ERANGE;   // the norm pass keeps K x 128 running sums in 48 KB of shared memory
+    if (ctx->cfg.K > 96) return QSR_ERANGE;   // the norm pass keeps K x kNormThreads running sums in 48 KB of shared memory
     ctx->clip_norm = max_norm; ctx->clip_ws = workspace_dev;
     return QSR_OK;
 }
@@ -329,10 +428,27 @@ int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
     for (int64_t t = t_begin; t < t_end;) {
         const int64_t H = qsr::round_length(ctx->cfg, t);       // GetH
         const RoundRange range(s, t, H);
-        for (int64_t h = 0; h + 1 < H; ++h)
+        const bool fuse_last = ctx->cfg.state_sync == QSR_STATE_KEEP;
+        int64_t h = 0;
+        if (graph_replay_applies(*ctx)) {
+            // whole segments of at most graph_steps launches; a round's tail takes its fused last step along
+            while (h < H) {
+                const int64_t left = H - h;
+                const bool tail = left <= ctx->graph_steps;
+                const int n_plain = int(tail ? left - 1 : ctx->graph_steps);
+                const bool fused = tail && fuse_last;
+                if (n_plain + (fused ? 1 : 0) == 0) break;      // only the unfused last step remains
+                const int rc = replay_steps(*ctx, t + h, n_plain, fused);
+                if (rc < 0) return rc;
+                if (rc > 0) break;                              // cache full: finish the round with direct launches
+                h += n_plain + (fused ? 1 : 0);
+            }
+        }
+        for (; h + 1 < H; ++h)
             if (int rc = qsr_local_step(ctx, t + h, nullptr)) return rc;
         // the round's last step and the parameter averaging, in one launch when the state is kept per worker
-        if (int rc = qsr_local_step_sync(ctx, t + H - 1, nullptr, t + H)) return rc;
+        if (h < H)
+            if (int rc = qsr_local_step_sync(ctx, t + H - 1, nullptr, t + H)) return rc;
         if (s < cap) {
             round_start[s] = t;
             round_len[s] = H;
@@ -341,6 +457,15 @@ int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
         t += H;
     }
     if (n_rounds) *n_rounds = s;
+    return QSR_OK;
+}
+
+int qsr_set_graph_replay(qsr_ctx *ctx, int32_t max_steps_per_graph)
+{
+    if (!ctx) return QSR_EINVAL;
+    if (max_steps_per_graph < 0 || max_steps_per_graph > 1024) return QSR_ERANGE;
+    if (max_steps_per_graph != ctx->graph_steps) drop_graphs(*ctx);
+    ctx->graph_steps = max_steps_per_graph;
     return QSR_OK;
 }
 
@@ -354,6 +479,7 @@ int qsr_set_launch_shape(qsr_ctx *ctx, int32_t step_threads, int32_t step_rows_i
     if (step_rows_in_flight != 0 && step_rows_in_flight != 1 && step_rows_in_flight != 2 && step_rows_in_flight != 4 &&
         step_rows_in_flight != 8)
         return QSR_ERANGE;
+    drop_graphs(*ctx);      // cached graphs carry the old geometry
     if (step_threads) ctx->shape.step_threads = step_threads;
     if (step_rows_in_flight) ctx->shape.step_rows = step_rows_in_flight;
     if (sync_threads) ctx->shape.sync_threads = sync_threads;
@@ -399,6 +525,9 @@ int qsr_train_host(const qsr_config *cfg, const float *theta0_host, const float 
 
     qsr_ctx *x = nullptr;
     if (int rc = qsr_init(&x, &c, theta, s1, s2, lambda, theta_star, cuda_stream)) return rc;
+    // Small problems are bound by launch overhead, not by memory: replay their rounds from CUDA graphs.
+    const int64_t bytes_per_step = 2 * int64_t(1 + n_state_slabs(c)) * slab * int64_t(sizeof(float));
+    if (bytes_per_step <= (int64_t(32) << 20)) qsr_set_graph_replay(x, 64);
     int rc = qsr_set_params(x, theta0);
     if (rc == QSR_OK) rc = qsr_run(x, 0, t_end, round_start, round_len, cap, n_rounds);
     if (rc == QSR_OK && cudaMemcpyAsync(theta_out_host, theta, row_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)

@@ -2,6 +2,7 @@
 #ifndef QSR_INTERNAL_H_
 #define QSR_INTERNAL_H_
 
+#include <cstddef>
 #include <cstdint>
 
 #include "../../include/qsr.h"
@@ -38,6 +39,7 @@ struct StepParams {
 };
 
 constexpr int kNormGrid = 1184;    // blocks of the gradient-norm pass (8 per SM on a 148-SM part)
+constexpr int kNormThreads = 128;  // its block size: K x 128 running sums must fit 48 KB of shared memory (K <= 96)
 
 struct SyncParams {
     float *slab[3];           // arrays to average (theta first), then arrays to zero
@@ -51,13 +53,28 @@ struct SyncParams {
 };
 
 struct LaunchShape {
-    // Defaults from sustained sweeps on B200 at the ViT-B/16 and ResNet-152 shapes (K = 16): 256-thread blocks with
-    // an 8-row cp.async ring per thread.  Grids capped at a few CTAs per SM with a grid-stride loop were 15-30 %
-    // slower than one thread per column.
+    // Defaults from sustained sweeps on B200 at the ViT-B/16 and ResNet-152 shapes (K = 16): an 8-row cp.async ring
+    // per thread, in 256-thread blocks for AdamW (96 KiB of ring, two blocks per SM) and 128-thread blocks for SGD
+    // (32 KiB, 0.7 % faster there than 256; qsr_init picks).  Grids capped at a few CTAs per SM with a grid-stride loop
+    // were 15-30 % slower than one thread per column.
     int step_threads = 256;
     int step_rows = 0;        // rows in flight per thread (ring depth); 0 = default (8)
     int sync_threads = 128;
 };
+
+// How the step kernel ends: plainly, with the replica mean written to every row (a round's last step), or with the
+// row sums written to StepParams::sum_out (a round's last step when the workers are sharded over GPUs).
+enum { FUSE_NONE = 0, FUSE_MEAN = 1, FUSE_SUM = 2 };
+
+// One instance of the step kernel with its launch geometry: what cudaLaunchKernel or a CUDA-graph kernel node needs.
+// The kernel's only argument is a StepParams by value.
+struct StepLaunch {
+    const void *func;
+    unsigned grid;
+    int threads;
+    size_t smem;
+};
+int resolve_step(const StepParams &p, int opt, const LaunchShape &shape, int fuse, StepLaunch *out);
 
 // kernels.cu -- each returns a cudaError_t cast to int (0 = success) after enqueueing one kernel.
 int launch_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream);
@@ -70,7 +87,7 @@ int launch_sync_finish(const SyncParams &p, const LaunchShape &shape, void *stre
 int launch_broadcast(float *theta, const float *theta0, int64_t P, int64_t stride, int32_t K,
                      const LaunchShape &shape, void *stream);
 // Gradient clipping: grid of the norm pass and the two passes that leave the factors at ws + clip_grid(...) * rows.
-int clip_grid(int64_t P, int threads);
+int clip_grid(int64_t P);
 int launch_clip_coef(const StepParams &p, bool parallel, double max_norm, float *ws, const LaunchShape &shape, void *stream);
 // Both phases through the library's own static scratch; -1 if the sums exceed QSR_STATIC_SCRATCH_FLOATS.
 int launch_sync_static(const SyncParams &p, const LaunchShape &shape, void *stream);

@@ -32,13 +32,22 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, const uint32_t (&rk)[20]
     return c;
 }
 
-// sqrt.approx / rcp-based division: one special-function instruction each instead of the IEEE sequences (about 8 and
-// 10 instructions with a slow-path branch).  Measured on B200 over 2^24 inputs: relative error of sqrt.approx at most
-// 1.0e-7 (mean -1.2e-8), of __fdividef at most 1.5e-7 (mean 3e-12) -- a rounding-level change, far inside the parity bound.
+// Square root and reciprocal as ONE special-function instruction each.  The IEEE forms are sequences of about 8 and
+// 10 instructions with a slow-path branch, and even the .approx forms carry extra scaling code for subnormal
+// operands unless they are the flush-to-zero variants used here.  Flushing is harmless at both call sites: the
+// Box-Muller radicand lies in [1e-7, 34], and a second moment below 1e-38 has a square root far below eps either way.
+// Measured on B200 over 2^24 inputs: relative error of sqrt.approx at most 1.0e-7 (mean -1.2e-8), of the reciprocal
+// at most 1.5e-7 (mean 3e-12) -- rounding-level, far inside the parity bound.
 __device__ __forceinline__ float sqrt_fast(float x)
 {
     float y;
-    asm("sqrt.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_fast(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
 
@@ -132,14 +141,17 @@ __device__ __forceinline__ void opt_update(float &theta, float &a, float &b, flo
         a = fmaf(p.mu, a, g);              // heavy-ball buffer
         theta = fmaf(-p.eta, a, theta);
     } else {
-        a = fmaf(p.beta1, a, p.omb1 * g);
-        b = fmaf(p.beta2, b, p.omb2 * g * g);
+        // Moments in the interpolation form x <- x + (1 - beta)(y - x): a constant gradient is then a fixed point
+        // exactly (m = g, v = g^2), whereas beta*x + (1 - beta)*y with both factors rounded to fp32 has fixed point
+        // y * fl(1 - beta) / (1 - fl(beta)), off by 2e-7 for beta1 = 0.9 and 1.3e-5 for beta2 = 0.999.
+        a = fmaf(p.omb1, g - a, a);
+        b = fmaf(p.omb2, fmaf(g, g, -b), b);
         const float denom = fmaf(sqrt_fast(b), p.inv_sqrt_bc2, p.eps);
         // theta*(1 - eta*wd) - step_size*m/denom as ONE subtraction from theta.  Forming 1 - eta*wd in fp32 would
         // keep only ~2^-24 of absolute precision on a term of size eta*wd, and the product theta*(1 - eta*wd) has
         // near-ties that round the same way step after step when theta sits just above a power of two; both show up
         // as a drift of a few 1e-5 over thousands of small steps.  The decay and the update are summed first instead.
-        theta -= fmaf(wdv, theta, p.step_size * __fdividef(a, denom));
+        theta -= fmaf(wdv, theta, (p.step_size * a) * rcp_fast(denom));
     }
 }
 
@@ -198,7 +210,6 @@ __device__ __forceinline__ void cp_async_wait_all_but() { asm volatile("cp.async
 //
 // EXTRAS selects the build that honours the per-tensor weight-decay table and the clipping factors; the plain build
 // (no table, clipping off: every run of the paper's QSR experiments) does not carry their tests in the row loop.
-enum { FUSE_NONE = 0, FUSE_MEAN = 1, FUSE_SUM = 2 };
 
 template <int OPT, bool EXT_GRAD>
 struct StepOperands {
@@ -571,9 +582,10 @@ unsigned grid_for(int64_t P, int threads)
     return unsigned(blocks);
 }
 
-// Launches one instance; raises its dynamic shared-memory limit first (the ring exceeds the 48 KB default).
+// Picks one instance of the step kernel and its launch geometry; raises the instance's dynamic shared-memory limit
+// (the ring exceeds the 48 KB default).  Returns a cudaError_t as int.
 template <int OPT, bool EXT, int STAGES, int FUSE, bool EXTRAS>
-int launch_step_instance(const StepParams &p, unsigned grid, int threads, cudaStream_t st)
+int resolve_step_instance(const StepParams &p, int threads, StepLaunch *out)
 {
     const size_t smem = size_t(STAGES) * StepOperands<OPT, EXT>::kCount * threads * sizeof(float4);
     if (smem > 227 * 1024) return int(cudaErrorInvalidValue);
@@ -582,55 +594,76 @@ int launch_step_instance(const StepParams &p, unsigned grid, int threads, cudaSt
         if (cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)))
             return int(e);
     }
-    kernel<<<grid, threads, smem, st>>>(p);
-    return int(cudaGetLastError());
+    out->func = reinterpret_cast<const void *>(kernel);
+    out->grid = grid_for(p.P, threads);
+    out->threads = threads;
+    out->smem = smem;
+    return 0;
 }
 
 template <int OPT, bool EXT, int FUSE, bool EXTRAS>
-int launch_step_stages(const StepParams &p, const LaunchShape &s, cudaStream_t st)
+int resolve_step_stages(const StepParams &p, const LaunchShape &s, StepLaunch *out)
 {
-    const unsigned grid = grid_for(p.P, s.step_threads);
     switch (s.step_rows ? s.step_rows : 8) {
-    case 1: return launch_step_instance<OPT, EXT, 1, FUSE, EXTRAS>(p, grid, s.step_threads, st);
-    case 2: return launch_step_instance<OPT, EXT, 2, FUSE, EXTRAS>(p, grid, s.step_threads, st);
-    case 4: return launch_step_instance<OPT, EXT, 4, FUSE, EXTRAS>(p, grid, s.step_threads, st);
-    default: return launch_step_instance<OPT, EXT, 8, FUSE, EXTRAS>(p, grid, s.step_threads, st);
+    case 1: return resolve_step_instance<OPT, EXT, 1, FUSE, EXTRAS>(p, s.step_threads, out);
+    case 2: return resolve_step_instance<OPT, EXT, 2, FUSE, EXTRAS>(p, s.step_threads, out);
+    case 4: return resolve_step_instance<OPT, EXT, 4, FUSE, EXTRAS>(p, s.step_threads, out);
+    default: return resolve_step_instance<OPT, EXT, 8, FUSE, EXTRAS>(p, s.step_threads, out);
     }
 }
 
 template <int OPT, bool EXT, int FUSE>
-int launch_step_rows(const StepParams &p, const LaunchShape &s, cudaStream_t st)
+int resolve_step_extras(const StepParams &p, const LaunchShape &s, StepLaunch *out)
 {
-    if (p.n_tensors > 0 || p.clip_coef) return launch_step_stages<OPT, EXT, FUSE, true>(p, s, st);
-    return launch_step_stages<OPT, EXT, FUSE, false>(p, s, st);
+    if (p.n_tensors > 0 || p.clip_coef) return resolve_step_stages<OPT, EXT, FUSE, true>(p, s, out);
+    return resolve_step_stages<OPT, EXT, FUSE, false>(p, s, out);
 }
 
 template <int FUSE>
-int launch_step_any(const StepParams &p, int opt, const LaunchShape &shape, cudaStream_t st)
+int resolve_step_fuse(const StepParams &p, int opt, const LaunchShape &shape, StepLaunch *out)
 {
     const bool ext = p.grads != nullptr;
     if (opt == QSR_OPT_SGDM)
-        return ext ? launch_step_rows<QSR_OPT_SGDM, true, FUSE>(p, shape, st)
-                   : launch_step_rows<QSR_OPT_SGDM, false, FUSE>(p, shape, st);
-    return ext ? launch_step_rows<QSR_OPT_ADAMW, true, FUSE>(p, shape, st)
-               : launch_step_rows<QSR_OPT_ADAMW, false, FUSE>(p, shape, st);
+        return ext ? resolve_step_extras<QSR_OPT_SGDM, true, FUSE>(p, shape, out)
+                   : resolve_step_extras<QSR_OPT_SGDM, false, FUSE>(p, shape, out);
+    return ext ? resolve_step_extras<QSR_OPT_ADAMW, true, FUSE>(p, shape, out)
+               : resolve_step_extras<QSR_OPT_ADAMW, false, FUSE>(p, shape, out);
+}
+
+int launch_resolved(const StepParams &p, int opt, const LaunchShape &shape, int fuse, void *stream)
+{
+    StepLaunch L;
+    if (int rc = resolve_step(p, opt, shape, fuse, &L)) return rc;
+    void *args[] = {const_cast<StepParams *>(&p)};
+    return int(cudaLaunchKernel(L.func, dim3(L.grid), dim3(unsigned(L.threads)), args, L.smem,
+                                static_cast<cudaStream_t>(stream)));
 }
 
 }  // namespace
 
+int resolve_step(const StepParams &p, int opt, const LaunchShape &shape, int fuse, StepLaunch *out)
+{
+    switch (fuse) {
+    case FUSE_NONE: return resolve_step_fuse<FUSE_NONE>(p, opt, shape, out);
+    case FUSE_MEAN: return resolve_step_fuse<FUSE_MEAN>(p, opt, shape, out);
+    case FUSE_SUM: return resolve_step_fuse<FUSE_SUM>(p, opt, shape, out);
+    default: return int(cudaErrorInvalidValue);
+    }
+}
+
 int launch_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream)
 {
-    return launch_step_any<FUSE_NONE>(p, opt, shape, static_cast<cudaStream_t>(stream));
+    return launch_resolved(p, opt, shape, FUSE_NONE, stream);
 }
 
 int launch_step_mean(const StepParams &p, int opt, const LaunchShape &shape, void *stream)
 {
-    return launch_step_any<FUSE_MEAN>(p, opt, shape, static_cast<cudaStream_t>(stream));
+    return launch_resolved(p, opt, shape, FUSE_MEAN, stream);
 }
 
 int launch_step_sum(const StepParams &p, int opt, const LaunchShape &shape, void *stream)
 {
-    return launch_step_any<FUSE_SUM>(p, opt, shape, static_cast<cudaStream_t>(stream));
+    return launch_resolved(p, opt, shape, FUSE_SUM, stream);
 }
 
 int launch_parallel_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream)
@@ -648,9 +681,9 @@ int launch_parallel_step(const StepParams &p, int opt, const LaunchShape &shape,
     return int(cudaGetLastError());
 }
 
-int clip_grid(int64_t P, int threads)
+int clip_grid(int64_t P)
 {
-    const int64_t want = (((P + 3) >> 2) + threads - 1) / threads;
+    const int64_t want = (((P + 3) >> 2) + kNormThreads - 1) / kNormThreads;
     return int(want < kNormGrid ? (want < 1 ? 1 : want) : kNormGrid);
 }
 
@@ -658,9 +691,9 @@ int clip_grid(int64_t P, int threads)
 int launch_clip_coef(const StepParams &p, bool parallel, double max_norm, float *ws, const LaunchShape &shape, void *stream)
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int threads = shape.step_threads;
+    const int threads = kNormThreads;
     const int rows = parallel ? 1 : p.K;
-    const int grid = clip_grid(p.P, threads);
+    const int grid = clip_grid(p.P);
     const size_t smem = size_t(rows) * threads * sizeof(float);
     if (smem > 48 * 1024) return int(cudaErrorInvalidValue);
     const bool ext = p.grads != nullptr;
