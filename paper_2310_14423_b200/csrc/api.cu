@@ -525,9 +525,6 @@ int qsr_train_host(const qsr_config *cfg, const float *theta0_host, const float 
 
     qsr_ctx *x = nullptr;
     if (int rc = qsr_init(&x, &c, theta, s1, s2, lambda, theta_star, cuda_stream)) return rc;
-    // Small problems are bound by launch overhead, not by memory: replay their rounds from CUDA graphs.
-    const int64_t bytes_per_step = 2 * int64_t(1 + n_state_slabs(c)) * slab * int64_t(sizeof(float));
-    if (bytes_per_step <= (int64_t(32) << 20)) qsr_set_graph_replay(x, 64);
     int rc = qsr_set_params(x, theta0);
     if (rc == QSR_OK) rc = qsr_run(x, 0, t_end, round_start, round_len, cap, n_rounds);
     if (rc == QSR_OK && cudaMemcpyAsync(theta_out_host, theta, row_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
