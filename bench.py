@@ -45,7 +45,7 @@ L2_BYTES = 126e6
 # once, so traffic grows in proportion to K*P).  Valid only for the kernel source it was taken from: the hash covers
 # the noise generator, the optimizer update and local_step_kernel in csrc/kernels.cu.
 NCU_TRAFFIC = {
-    "step_source_sha256": "ff2976835143924ba17aaf60339c53736ec7b83cadb9db352fc744aec8fd6278",
+    "step_source_sha256": "6c2fa12f453d27aa841b9366d84720bff8d1390a3c74bc8ff30a60d58949601e",
     "bytes_per_update": {"adamw": 24.064, "sgdm": 16.069},
 }
 

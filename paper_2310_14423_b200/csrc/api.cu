@@ -228,6 +228,17 @@ int qsr_init(qsr_ctx **out, const qsr_config *cfg, float *params, float *state1,
     x->stream = static_cast<cudaStream_t>(cuda_stream);
     x->shape = qsr::LaunchShape();
     if (cfg->opt == QSR_OPT_SGDM) x->shape.step_threads = 128;
+    // Slabs that stay resident in L2 between steps are served with far lower latency than HBM: a 4-row ring in
+    // 128-thread blocks (more blocks per SM, shorter prologue) then beats the 8-row ring (K = 8, P = 2^20 AdamW on
+    // B200: 31.3 us against 35.7 us per step).
+    int l2_bytes = 0;
+    if (cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, dev) == cudaSuccess) {
+        const int64_t state_bytes = int64_t(1 + n_state_slabs(*cfg)) * cfg->K * cfg->row_stride * int64_t(sizeof(float));
+        if (state_bytes <= int64_t(l2_bytes) / 5 * 4) {
+            x->shape.step_threads = 128;
+            x->shape.step_rows = 4;
+        }
+    }
     x->t_state_origin = cfg->t_state_origin;
     x->launches = 0;
     x->partial_pending = false;

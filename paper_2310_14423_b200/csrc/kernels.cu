@@ -4,8 +4,8 @@
 // Both are pure HBM streams over [K, P] fp32 slabs: nothing here is a contraction, so there are no tensor-core
 // instructions.  A thread owns one 16-byte column (4 consecutive coordinates) for ALL K rows: lambda / theta_star
 // are fetched once per column instead of once per worker, every global access is a 128-bit LDG/STG on a
-// 16-byte boundary, a warp touches 512 contiguous bytes per row, and the loads of several rows are issued before
-// the first use so that each SM keeps enough bytes in flight to cover HBM latency.
+// 16-byte boundary, a warp touches 512 contiguous bytes per row, and the step kernel keeps the loads of eight rows
+// per thread in flight through a cp.async ring in shared memory to cover HBM latency.
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -197,7 +197,8 @@ __device__ __forceinline__ void cp_async_wait_all_but() { asm volatile("cp.async
 // memory; the ring is filled STAGES rows ahead, and as soon as a row has been copied to registers its slot is
 // refilled with row k + STAGES.  With 256 threads, 8 stages and AdamW's three operands a CTA holds 96 KB of loads in
 // flight (two CTAs per SM), against about 60 KB per SM when the rows in flight had to live in registers; on B200
-// that took the ViT-B/16-shaped AdamW step from 5.58 ms to 5.31 ms (6.38 TB/s, 99 % of a device copy).
+// that took the sustained ViT-B/16-shaped AdamW step from 5.6 ms to 5.35 ms, and trimming the instruction stream
+// (see the noise section) brought it to 5.3 ms, 97-98 % of the rate of a device-to-device copy.
 // Results go straight from registers to global memory with 128-bit stores.
 //
 // Round end.  With FUSE != 0 the step is the last of its round and the kernel also ends the round (Algorithm 2's
