@@ -232,11 +232,12 @@ def main():
     ths = torch.zeros(P4, device=dev)
     lam[:w.P].copy_(torch.from_numpy(lam_h))
     ths[:w.P].copy_(torch.from_numpy(ths_h))
-    theta = torch.zeros(K_local, P4, device=dev)
-    s1 = torch.zeros(K_local, P4, device=dev)
-    s2 = torch.zeros(K_local, P4, device=dev) if w.opt == W.OPT_ADAMW else None
+    stride = B.qsr_row_stride_hint(w.P)       # rows on large power-of-two boundaries: see include/qsr.h
+    theta = torch.zeros(K_local, stride, device=dev)
+    s1 = torch.zeros(K_local, stride, device=dev)
+    s2 = torch.zeros(K_local, stride, device=dev) if w.opt == W.OPT_ADAMW else None
     stream = torch.cuda.current_stream().cuda_stream
-    cfg = B.make_config(w, K=K_local, row_stride=P4)
+    cfg = B.make_config(w, K=K_local, row_stride=stride)
     sharded_path = world > 1 or args.sharded_path      # rounds end with partial sums + all-reduce + finish
     sums = torch.zeros(3 * P4, device=dev) if sharded_path else None
 
@@ -431,7 +432,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": label, "K_per_gpu": K_local, "K_total": K_total, "P": w.P, "opt": w.opt, "T": w.T,
+        "config": {"workload": label, "K_per_gpu": K_local, "K_total": K_total, "P": w.P, "row_stride": stride, "opt": w.opt, "T": w.T,
                    "window": f"global steps [0,{steps}) of the schedule", "syncs_in_window": n_syncs,
                    "l2": l2_note,
                    "parallelism": f"replica-sharded dp{world}" if sharded_path else "1 GPU, replicas as slab rows"},

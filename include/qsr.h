@@ -110,6 +110,15 @@ int64_t qsr_config_round_length(const qsr_config *cfg, int64_t t);
  * qsr_status.  The share of steps that synchronize (the "Comm." column of Tables 1-3) is rounds / T. */
 int64_t qsr_config_schedule(const qsr_config *cfg, int64_t *round_start, int64_t *round_len, int64_t cap);
 
+/* A row stride (in floats, a multiple of 4, >= P) that lets the kernels stream at full rate.  Any stride that obeys
+ * the conventions above is legal, but where the K rows of a slab start matters to the memory system: on B200, with
+ * K = 16 rows of P = 86,415,592 floats packed at P, the AdamW step takes 5.33 ms; with every row on a 16 KiB boundary
+ * 5.19 ms, on a 256 KiB boundary 5.16 ms, on a 4 MiB boundary 5.12 ms (the averaging kernel 1.77 -> 1.68 ms; K = 32:
+ * 10.76 -> 10.26 ms).  The hint rounds P up to a multiple of 2^a floats, a = min(20, floor(log2 P) - 4) but at least
+ * 2, so the padding stays below P/16 (at most 4 MiB per row); padding is never read or written.  Negative qsr_status
+ * if P < 1. */
+int64_t qsr_row_stride_hint(int64_t P);
+
 /* Bytes of device workspace that qsr_train_host needs for cfg (slabs plus the two input vectors). */
 int64_t qsr_workspace_bytes(const qsr_config *cfg);
 
@@ -253,7 +262,7 @@ int qsr_set_launch_shape(qsr_ctx *ctx, int32_t step_threads, int32_t step_rows_i
  * worker a copy of theta0, zeroes the optimizer state, runs steps [0, t_end) as qsr_run does, copies worker 0's
  * parameters (all workers are equal after the last synchronization) to theta_out_host [P], and waits for the
  * stream.  workspace_dev: caller-owned device memory of at least qsr_workspace_bytes(cfg) bytes, 256-byte aligned.
- * cfg->row_stride is ignored (rows are packed at P rounded up to 4).  round_* / n_rounds as in qsr_run;
+ * cfg->row_stride is ignored (rows are laid out at qsr_row_stride_hint(P)).  round_* / n_rounds as in qsr_run;
  * *launches (may be NULL) receives the number of kernel launches. */
 int qsr_train_host(const qsr_config *cfg, const float *theta0_host, const float *lambda_host,
                    const float *theta_star_host, float *theta_out_host,

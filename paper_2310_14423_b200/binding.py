@@ -25,7 +25,7 @@ STATE = {"keep": 0, "average": 1, "reset": 2}
 QSR_OK, QSR_EINVAL, QSR_EALIGN, QSR_ECUDA, QSR_ERANGE, QSR_ESTATE = 0, -1, -2, -3, -4, -5
 QSR_STATIC_SCRATCH_FLOATS = 1 << 20
 
-EXPORTS = ("qsr_config_check", "qsr_config_learning_rate", "qsr_config_round_length", "qsr_config_schedule",
+EXPORTS = ("qsr_config_check", "qsr_row_stride_hint", "qsr_config_learning_rate", "qsr_config_round_length", "qsr_config_schedule",
            "qsr_workspace_bytes", "qsr_init", "qsr_destroy", "qsr_round_length", "qsr_set_tensor_table", "qsr_clip_workspace_floats", "qsr_set_grad_clip", "qsr_set_params", "qsr_local_step",
            "qsr_local_step_sync", "qsr_parallel_step", "qsr_sync", "qsr_sync_sum_floats", "qsr_sync_partial", "qsr_local_step_partial", "qsr_sync_finish", "qsr_sync_static", "qsr_run", "qsr_launch_count",
            "qsr_set_launch_shape", "qsr_set_graph_replay", "qsr_train_host", "qsr_strerror")
@@ -63,6 +63,7 @@ def lib():
         cfg, vp, i64, i32 = C.POINTER(QsrConfig), C.c_void_p, C.c_int64, C.c_int32
         sig = {
             "qsr_config_check": (C.c_int, [cfg]),
+            "qsr_row_stride_hint": (i64, [i64]),
             "qsr_config_learning_rate": (C.c_double, [cfg, i64]),
             "qsr_config_round_length": (i64, [cfg, i64]),
             "qsr_config_schedule": (i64, [cfg, vp, vp, i64]),
@@ -146,6 +147,13 @@ def qsr_config_schedule(cfg: QsrConfig) -> Tuple[np.ndarray, np.ndarray]:
     if n < 0:
         raise QsrError(n, "qsr_config_schedule")
     return st[:n].copy(), H[:n].copy()
+
+
+def qsr_row_stride_hint(P: int) -> int:
+    n = int(lib().qsr_row_stride_hint(int(P)))
+    if n < 0:
+        raise QsrError(n, "qsr_row_stride_hint")
+    return n
 
 
 def qsr_workspace_bytes(cfg: QsrConfig) -> int:

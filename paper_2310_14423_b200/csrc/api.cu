@@ -501,7 +501,7 @@ int64_t qsr_workspace_bytes(const qsr_config *cfg)
 {
     if (!cfg) return QSR_EINVAL;
     qsr_config c = *cfg;
-    c.row_stride = round_up4(c.P);
+    c.row_stride = qsr::row_stride_hint(c.P);
     if (int rc = qsr::check_config(c)) return rc;
     const int64_t slabs = 1 + n_state_slabs(c);
     return (slabs * c.K * c.row_stride + 3 * c.row_stride) * int64_t(sizeof(float));
@@ -514,7 +514,7 @@ int qsr_train_host(const qsr_config *cfg, const float *theta0_host, const float 
 {
     if (!cfg || !theta0_host || !lambda_host || !theta_star_host || !theta_out_host || !workspace_dev) return QSR_EINVAL;
     qsr_config c = *cfg;
-    c.row_stride = round_up4(c.P);
+    c.row_stride = qsr::row_stride_hint(c.P);
     c.t_state_origin = 0;
     if (int rc = qsr::check_config(c)) return rc;
     if ((reinterpret_cast<uintptr_t>(workspace_dev) & 255u) != 0) return QSR_EALIGN;

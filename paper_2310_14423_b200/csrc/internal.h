@@ -11,6 +11,7 @@ namespace qsr {
 
 // schedule.cpp
 int check_config(const qsr_config &c);
+int64_t row_stride_hint(int64_t P);
 double learning_rate(const qsr_config &c, int64_t t);
 int64_t round_length(const qsr_config &c, int64_t t);
 

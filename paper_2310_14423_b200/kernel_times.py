@@ -19,6 +19,8 @@ def main(argv=None):
     ap.add_argument("--workload", default="c4")
     ap.add_argument("--launches", type=int, default=30)
     ap.add_argument("--out", default=None)
+    ap.add_argument("--packed", action="store_true",
+                    help="rows packed at P instead of the stride qsr_row_stride_hint recommends")
     args = ap.parse_args(argv)
 
     import torch
@@ -31,7 +33,8 @@ def main(argv=None):
     w = W.workload(args.workload)
     KP = w.K * w.P
     n_slabs = 3 if w.opt == W.OPT_ADAMW else 2
-    theta = torch.zeros(w.K, w.P, device=dev)
+    stride = (w.P + 3) // 4 * 4 if args.packed else B.qsr_row_stride_hint(w.P)
+    theta = torch.zeros(w.K, stride, device=dev)
     s1 = torch.zeros_like(theta)
     s2 = torch.zeros_like(theta) if w.opt == W.OPT_ADAMW else None
     lam = torch.rand(w.P, device=dev)
@@ -52,7 +55,7 @@ def main(argv=None):
         return e0.elapsed_time(e1) / args.launches
 
     def context(mode=W.STATE_KEEP):
-        return B.Context(B.make_config(w.replace(state_sync=mode)), theta, s1, s2, lam, ths, stream=stream)
+        return B.Context(B.make_config(w.replace(state_sync=mode), row_stride=stride), theta, s1, s2, lam, ths, stream=stream)
 
     rows = []
 
@@ -110,7 +113,7 @@ def main(argv=None):
         c = context(mode)
         add(f"replica mean, state {mode}", timed(lambda: c.qsr_sync(t[0])), per * KP)
         c.close()
-    theta0 = torch.zeros(w.P, device=dev)
+    theta0 = torch.zeros(stride, device=dev)[:w.P]
     c = context()
     add("broadcast of theta_bar(0) to every worker", timed(lambda: c.qsr_set_params(theta0)), 4 * KP + 4 * w.P)
     c.close()

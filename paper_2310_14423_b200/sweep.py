@@ -39,7 +39,8 @@ def main(argv=None):
     ths = torch.zeros(P4, device=dev)
     lam[:base.P].copy_(torch.from_numpy(lam_h))
     ths[:base.P].copy_(torch.from_numpy(ths_h))
-    theta = torch.zeros(base.K, P4, device=dev)
+    stride = B.qsr_row_stride_hint(base.P)
+    theta = torch.zeros(base.K, stride, device=dev)
     s1 = torch.zeros_like(theta)
     s2 = torch.zeros_like(theta) if base.opt == W.OPT_ADAMW else None
     stream = torch.cuda.current_stream().cuda_stream
@@ -56,7 +57,7 @@ def main(argv=None):
     lines = ["| eta_max | setting | rounds (syncs) | comm. % | launches | total s | ms / step | param-updates / s |",
              "|---|---|---|---|---|---|---|---|"]
     for label, w in settings:
-        cfg = B.make_config(w, row_stride=P4)
+        cfg = B.make_config(w, row_stride=stride)
         st, H = B.qsr_config_schedule(cfg)
         t_end = w.T if args.steps is None else min(w.T, args.steps)
         key = (w.eta_max, tuple(H[st < t_end].tolist()))

@@ -110,7 +110,27 @@ def test_workspace_bytes():
     cfg = B.make_config(w)
     assert B.qsr_workspace_bytes(cfg) == (3 * w.K * w.P + 3 * w.P) * 4
     w = W.tiny_workload(W.OPT_SGDM, K=3, P=1001)
-    assert B.qsr_workspace_bytes(B.make_config(w)) == (2 * 3 * 1004 + 3 * 1004) * 4
+    stride = B.qsr_row_stride_hint(1001)
+    assert stride == 1024
+    assert B.qsr_workspace_bytes(B.make_config(w)) == (2 * 3 * stride + 3 * stride) * 4
+
+
+def test_row_stride_hint():
+    """A legal stride (multiple of 4, >= P) on a power-of-two boundary of at most 2^20 floats, padding below P/16."""
+    for P in (1, 2, 3, 4, 5, 63, 64, 65, 1000, 65535, 65536, 65537, 1 << 20, (1 << 20) + 1, 60_192_808, 86_415_592,
+              (1 << 31) + 12345):
+        s = B.qsr_row_stride_hint(P)
+        assert s >= P and s % 4 == 0
+        unit = s & -s                        # largest power of two dividing the stride
+        assert s - P < max(4, P / 16)
+        assert unit >= min(1 << 20, max(4, 1 << max(0, P.bit_length() - 5)))
+        cfg = B.make_config(W.tiny_workload(W.OPT_SGDM, K=2, P=P), row_stride=s)
+        assert B.qsr_config_check(cfg) == B.QSR_OK
+    assert B.qsr_row_stride_hint(86_415_592) == 83 * (1 << 20)
+    for bad in (0, -7):
+        with pytest.raises(B.QsrError) as e:
+            B.qsr_row_stride_hint(bad)
+        assert e.value.status == B.QSR_EINVAL
 
 
 def _same_schedule(w):

@@ -21,10 +21,11 @@ N_SUBSET = 4096
 
 def _run_device(w, t_end=None):
     lam, ths, lam_d, ths_d = G.device_inputs(w)
-    theta = torch.zeros(w.K, w.P, device="cuda")
-    s1 = torch.zeros(w.K, w.P, device="cuda")
-    s2 = torch.zeros(w.K, w.P, device="cuda") if w.opt == W.OPT_ADAMW else None
-    cfg = B.make_config(w)
+    stride = B.qsr_row_stride_hint(w.P)              # the layout bench.py uses
+    theta = torch.zeros(w.K, stride, device="cuda")
+    s1 = torch.zeros(w.K, stride, device="cuda")
+    s2 = torch.zeros(w.K, stride, device="cuda") if w.opt == W.OPT_ADAMW else None
+    cfg = B.make_config(w, row_stride=stride)
     ctx = B.Context(cfg, theta, s1, s2, lam_d, ths_d, stream=torch.cuda.current_stream().cuda_stream)
     st, H = ctx.qsr_run(0, t_end)
     torch.cuda.synchronize()
@@ -87,4 +88,4 @@ def test_k32_slab_beyond_32bit_indexing():
     lam, ths, theta, st, H = _run_device(w, t_end=500)
     assert st.tolist() == [0, 478] and H.tolist() == [478, 481]
     _compare(w, lam, ths, theta, st, H, t_end=500)
-    assert bool((theta[31] == theta[0]).all())
+    assert bool((theta[31, :w.P] == theta[0, :w.P]).all())
