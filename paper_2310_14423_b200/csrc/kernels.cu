@@ -441,36 +441,21 @@ __global__ void grad_sqnorm_kernel(const __grid_constant__ StepParams p, float *
             lam = ld4_guarded(p.lambda + i0, valid);     // zero lambda and zero noise weight make the lanes beyond P vanish
             ths = ld4_guarded(p.theta_star + i0, valid);
         }
-        for (int k0 = 0; k0 < p.K; k0 += 8) {
-            // the operand rows of eight workers (their gradients, or the parameters the gradients are generated from):
-            // all loads are issued before the first use
-            float4 v[8];
-#pragma unroll
-            for (int r = 0; r < 8; ++r) {
-                if (k0 + r < p.K) {
-                    // Algorithm 1 evaluates every worker's gradient at the single model in row 0
-                    const float *row = EXT_GRAD ? p.grads + int64_t(k0 + r) * p.stride
-                                                : p.theta + int64_t(PARALLEL ? 0 : k0 + r) * p.stride;
-                    v[r] = ld4_guarded(row + i0, valid);
-                }
+        for (int k = 0; k < p.K; ++k) {
+            float4 g;
+            if (EXT_GRAD) {
+                g = ld4_guarded(p.grads + int64_t(k) * p.stride + i0, valid);
+            } else {
+                // Algorithm 1 evaluates every worker's gradient at the single model in row 0
+                const float4 th = ld4_guarded(p.theta + int64_t(PARALLEL ? 0 : k) * p.stride + i0, valid);
+                const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.round_key);
+                g.x = fmaf(p.sigma, z.x, lam.x * (th.x - ths.x));
+                g.y = valid > 1 ? fmaf(p.sigma, z.y, lam.y * (th.y - ths.y)) : 0.f;
+                g.z = valid > 2 ? fmaf(p.sigma, z.z, lam.z * (th.z - ths.z)) : 0.f;
+                g.w = valid > 3 ? fmaf(p.sigma, z.w, lam.w * (th.w - ths.w)) : 0.f;
             }
-#pragma unroll
-            for (int r = 0; r < 8; ++r) {
-                const int k = k0 + r;
-                if (k < p.K) {
-                    float4 g = v[r];
-                    if (!EXT_GRAD) {
-                        const float4 th = v[r];
-                        const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.round_key);
-                        g.x = fmaf(p.sigma, z.x, lam.x * (th.x - ths.x));
-                        g.y = valid > 1 ? fmaf(p.sigma, z.y, lam.y * (th.y - ths.y)) : 0.f;
-                        g.z = valid > 2 ? fmaf(p.sigma, z.z, lam.z * (th.z - ths.z)) : 0.f;
-                        g.w = valid > 3 ? fmaf(p.sigma, z.w, lam.w * (th.w - ths.w)) : 0.f;
-                    }
-                    if (PARALLEL) sum = add4(sum, g);
-                    else acc[k * blockDim.x + threadIdx.x] += (g.x * g.x + g.y * g.y) + (g.z * g.z + g.w * g.w);
-                }
-            }
+            if (PARALLEL) sum = add4(sum, g);
+            else acc[k * blockDim.x + threadIdx.x] += (g.x * g.x + g.y * g.y) + (g.z * g.z + g.w * g.w);
         }
         if (PARALLEL) {
             sum = div4(sum, Kf);
