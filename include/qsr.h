@@ -115,8 +115,10 @@ int64_t qsr_config_schedule(const qsr_config *cfg, int64_t *round_start, int64_t
  * K = 16 rows of P = 86,415,592 floats packed at P, the AdamW step takes 5.33 ms; with every row on a 16 KiB boundary
  * 5.19 ms, on a 256 KiB boundary 5.16 ms, on a 4 MiB boundary 5.12 ms (the averaging kernel 1.77 -> 1.68 ms; K = 32:
  * 10.76 -> 10.26 ms).  The hint rounds P up to a multiple of 2^a floats, a = min(20, floor(log2 P) - 4) but at least
- * 2, so the padding stays below P/16 (at most 4 MiB per row); padding is never read or written.  Negative qsr_status
- * if P < 1. */
+ * 2, so the padding stays below P/16 (at most 4 MiB per row); padding is never read or written.  The base addresses
+ * of params / state1 / state2 should agree modulo 4 KiB as well (state slabs shifted by 128 bytes against params cost
+ * 1.6 %; shifts of 4 KiB and more cost nothing); large blocks from cudaMalloc or a caching allocator do.  Negative
+ * qsr_status if P < 1. */
 int64_t qsr_row_stride_hint(int64_t P);
 
 /* Bytes of device workspace that qsr_train_host needs for cfg (slabs plus the two input vectors). */
