@@ -59,6 +59,8 @@ def parse_args():
     ap.add_argument("--workload", default="c4")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--packed-rows", action="store_true",
+                    help="rows packed at P (rounded up to 4) instead of the stride qsr_row_stride_hint recommends")
     ap.add_argument("--sharded-path", action="store_true",
                     help="on one GPU, still end rounds the multi-GPU way (partial sums, all-reduce of one rank, finish)")
     return ap.parse_args()
@@ -232,7 +234,8 @@ def main():
     ths = torch.zeros(P4, device=dev)
     lam[:w.P].copy_(torch.from_numpy(lam_h))
     ths[:w.P].copy_(torch.from_numpy(ths_h))
-    stride = B.qsr_row_stride_hint(w.P)       # rows on large power-of-two boundaries: see include/qsr.h
+    # rows on large power-of-two boundaries (see include/qsr.h) unless asked to pack them
+    stride = P4 if args.packed_rows else B.qsr_row_stride_hint(w.P)
     theta = torch.zeros(K_local, stride, device=dev)
     s1 = torch.zeros(K_local, stride, device=dev)
     s2 = torch.zeros(K_local, stride, device=dev) if w.opt == W.OPT_ADAMW else None

@@ -195,6 +195,10 @@ def workload(name: str) -> Workload:
     c4p as c4 with the paper's peak lr 0.008 (App. C.2), so that H_base shapes the schedule
     c5  K=32, ViT-B/16 shapes (sweep base: alpha, H_base and the rule are overridden by the caller)
     """
+    if name == "c4u":
+        # c4s with eight more parameters: rows of 2^25 + 32 bytes, so that rows packed at P start at unrelated offsets
+        # of every power-of-two address unit, as the rows of the full-size shaped sets do.
+        return workload("c4").replace(name=name, layout=flat_layout((1 << 23) + 8))
     if name in ("c3s", "c4s", "c4ps"):
         # The same runs on a flat 2^23-parameter set: slabs of 512 MiB, larger than L2 but small enough for
         # profiler captures that replay each launch many times.
