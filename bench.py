@@ -92,6 +92,7 @@ class ClockSampler:
               "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_id: str):
+        self.gpu_id = gpu_id
         self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", gpu_id, f"--query-gpu={self.FIELDS}",
@@ -111,9 +112,19 @@ class ClockSampler:
             self.proc.kill()
         self.tmp.flush()
         self.tmp.seek(0)
+        lines = self.tmp.readlines()
+        late = not lines
+        if late:
+            # the timed region ended before the first 200 ms sample: take one reading now
+            try:
+                lines = subprocess.run(["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.FIELDS}",
+                                        "--format=csv,noheader,nounits"], capture_output=True, text=True,
+                                       timeout=20).stdout.splitlines()
+            except Exception:
+                lines = []
         sm, smax, power, reasons = [], [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in self.tmp:
+        for line in lines:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 8:
                 continue
@@ -131,6 +142,8 @@ class ClockSampler:
         if sm:
             out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(smax)), reasons=sorted(reasons),
                        samples=len(sm), power_w_median=float(np.median(power)))
+            if late:
+                out["note"] = "one reading taken right after the timed region, which was shorter than the sampling period"
         return out
 
 
