@@ -317,6 +317,24 @@ def test_fused_last_step_equals_step_then_sync_bitwise(opt, K, P):
     cb.close()
 
 
+@pytest.mark.parametrize("opt", [W.OPT_SGDM, W.OPT_ADAMW])
+def test_row_stride_does_not_change_the_bits(opt):
+    """Rows packed at P, at the stride the library recommends and at an odd padded stride: the layout is a matter of
+    speed only, every parameter and state value is bit-identical (padding stays untouched: the guards check it)."""
+    w = W.tiny_workload(opt, K=5, P=70003, T=60)
+    hinted = B.qsr_row_stride_hint(w.P)
+    assert hinted % 4096 == 0 and hinted >= w.P
+    runs = []
+    for stride in ((w.P + 3) // 4 * 4, hinted, (w.P + 3) // 4 * 4 + 36):
+        lam, ths, S, st, H, _ = _run_full(w, row_stride=stride)
+        assert S.guards_intact()
+        runs.append(S)
+    for S in runs[1:]:
+        assert torch.equal(S.theta[:, :w.P], runs[0].theta[:, :w.P])
+        assert torch.equal(S.s1[:, :w.P], runs[0].s1[:, :w.P])
+        assert S.s2 is None or torch.equal(S.s2[:, :w.P], runs[0].s2[:, :w.P])
+
+
 def test_nonzero_start_and_set_params():
     w = W.tiny_workload(W.OPT_SGDM, K=3, P=999, T=30)
     lam, ths, lam_d, ths_d = G.device_inputs(w)
