@@ -13,6 +13,7 @@
  *     allocates no device memory and frees none.  Pointers with "host" in their name are HOST pointers.
  *   - Slabs are row-major [K, row_stride] floats; worker k's coordinate i is slab[k * row_stride + i],
  *     i < P <= row_stride, row_stride a multiple of 4.  Elements with i >= P are never read or written.
+ *     Any such stride works; qsr_row_stride_hint(P) is the one the kernels stream fastest with.
  *   - Device work is enqueued on the CUDA stream given to qsr_init; no call waits for the device except
  *     qsr_train_host.  The host-side schedule functions do no device work at all.
  *   - Every function returns QSR_OK (0) or a negative qsr_status; none aborts, throws or exits.  A failed
