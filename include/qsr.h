@@ -218,8 +218,11 @@ int qsr_sync_finish(qsr_ctx *ctx, const float *sum, int32_t K_total, int64_t t_n
  *   - The sums must fit: (P rounded up to 4) floats, times 1 + the number of state slabs in AVERAGE mode, must not
  *     exceed QSR_STATIC_SCRATCH_FLOATS.  Larger problems get QSR_ERANGE and nothing is launched; use qsr_sync, or
  *     qsr_sync_partial / qsr_sync_finish with a buffer of your own.
- *   - The first call on a device looks up the array's device address (once per device; the context's device must be
- *     current, as for every call).  Make that first call before any stream capture begins.
+ *   - The first call on a device looks up the array's device address (once per device) and keeps it for the life of
+ *     the process.  Make that first call before any stream capture begins.  The device the context was created on
+ *     must be current (QSR_ESTATE otherwise, nothing launched).  Contexts on different host threads may make their
+ *     first calls at the same time.  cudaDeviceReset destroys the array the kept address points to: do not call
+ *     qsr_sync_static in a process that has reset the device after using it.
  *   - All contexts and all calls in the process share the one array.  Each call overwrites what it needs before
  *     reading it, so an earlier call's leftovers are harmless; but two calls whose kernels can overlap on the GPU
  *     (different streams, no ordering between them) race on it.  Keep the calls on one stream or order them.
@@ -271,6 +274,18 @@ int qsr_train_host(const qsr_config *cfg, const float *theta0_host, const float 
                    const float *theta_star_host, float *theta_out_host,
                    void *workspace_dev, int64_t workspace_bytes, int64_t t_end, void *cuda_stream,
                    int64_t *round_start, int64_t *round_len, int64_t cap, int64_t *n_rounds, int64_t *launches);
+
+/* ---- test hook ---------------------------------------------------------------------------------------- */
+
+/* The two halves of the Box-Muller transform that turns generator words into the synthetic gradient's noise (the
+ * stand-in for Sample() and back-propagation in Algorithm 2; formula at qsr_config), evaluated by the same device
+ * code the step kernels inline.  For each of the n words w in words_dev (device, uint32), with the 23-bit field
+ * a = w >> 9 and u = (a + 1/2) / 2^23:  radius_dev[i] = sqrt(-2 ln u), sin_dev[i] = sin(2 pi u), cos_dev[i] = cos(2 pi u)
+ * (device, float, n each; 4-byte aligned).  A step uses the radius of one word with the sine / cosine of the next.
+ * The field has only 2^23 values, so a test can compare every one with binary64.  No context; one launch on
+ * cuda_stream; asynchronous.  QSR_EINVAL for n < 0 or a NULL array with n > 0. */
+int qsr_debug_box_muller(const uint32_t *words_dev, int64_t n, float *radius_dev, float *sin_dev, float *cos_dev,
+                         void *cuda_stream);
 
 /* Text for a qsr_status. Never NULL. */
 const char *qsr_strerror(int status);

@@ -31,8 +31,15 @@
  *                     samples mini-batches; the synthetic workload replaces fwd/bwd by a diagonal
  *                     quadratic loss plus this noise.
  *
- * Arithmetic is binary64 throughout (build with -DORC_REAL=float for the "mirror" build, which
- * keeps the same order of operations in binary32 and serves only to size rounding error).
+ * Arithmetic is binary64 throughout.  Built with -DORC_REAL=float the same file gives the "mirror", a
+ * yardstick for what binary32 costs on a given run: parameters, optimizer state, gradients and means
+ * are STORED in binary32 and the synthetic gradient lambda*(theta - theta_star) + sigma*z is evaluated
+ * in binary32 (its cancellation is the one ill-conditioned spot of the path, and it is there for any
+ * implementation that keeps the gradient in fp32), while the optimizer update and the mean are
+ * evaluated in binary64 from the stored values and rounded once when they are stored.  The mirror's
+ * distance from the binary64 build is therefore close to the least error an fp32 path can have on that
+ * run, and it is large exactly where the run is ill-conditioned.  In the binary64 build every cast to
+ * `real` is a no-op.
  *
  * Parity pins (tests/test_oracle_*.py): the schedule against the communication volumes the paper
  * prints in Tables 1-3 and against threshold crossings derived by inverting the cosine; SGD against
@@ -178,14 +185,33 @@ void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
+/* The two halves of the Box-Muller transform on the 23-bit fields a and b of two generator words: the
+ * uniforms are u1 = (a + 1/2) / 2^23 and u2 = (b + 1/2) / 2^23, which lie strictly inside (0,1) and are
+ * exact in binary32 and binary64; radius = sqrt(-2 ln u1), and the sine and cosine of the angle 2 pi u2. */
+void orc_box_muller_parts(uint32_t a, uint32_t b, double *radius, double *sine, double *cosine)
+{
+    const double two_pi = 6.28318530717958647692;
+    double u1 = ((double)a + 0.5) / 8388608.0;
+    double u2 = ((double)b + 0.5) / 8388608.0;
+    *radius = sqrt(-2.0 * log(u1));
+    *sine = sin(two_pi * u2);
+    *cosine = cos(two_pi * u2);
+}
+
+/* The same for arrays of fields: a convenience for tests that walk the whole 23-bit grid. */
+void orc_box_muller_parts_fill(const uint32_t *a, const uint32_t *b, int64_t n, double *radius, double *sine, double *cosine)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t c = 0; c < n; ++c)
+        orc_box_muller_parts(a[c], b[c], radius + c, sine + c, cosine + c);
+}
+
 /* Standard normal for (seed, worker k, global step u, coordinate i).
  * One Philox block serves coordinates 4j..4j+3: counter = (low(j), high(j), u, k), key = seed.
  * Words (0,1) feed the Box-Muller pair for coordinates 4j (cosine branch) and 4j+1 (sine branch),
- * words (2,3) the pair for 4j+2 and 4j+3.  Each word gives a 23-bit field a; the uniform is
- * (a + 1/2) / 2^23, which lies strictly inside (0,1) and is exact in binary32 and binary64. */
+ * words (2,3) the pair for 4j+2 and 4j+3.  Each word gives a 23-bit field (its top 23 bits). */
 double orc_noise(uint64_t seed, int64_t k, int64_t u, int64_t i)
 {
-    const double two_pi = 6.28318530717958647692;
     uint64_t j = (uint64_t)i >> 2;
     uint32_t ctr[4] = { (uint32_t)j, (uint32_t)(j >> 32), (uint32_t)u, (uint32_t)k };
     uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
@@ -194,15 +220,15 @@ double orc_noise(uint64_t seed, int64_t k, int64_t u, int64_t i)
     int lane = (int)(i & 3);
     uint32_t a = r[(lane >> 1) * 2] >> 9;
     uint32_t b = r[(lane >> 1) * 2 + 1] >> 9;
-    double u1 = ((double)a + 0.5) / 8388608.0;
-    double u2 = ((double)b + 0.5) / 8388608.0;
-    double radius = sqrt(-2.0 * log(u1));
-    return (lane & 1) ? radius * sin(two_pi * u2) : radius * cos(two_pi * u2);
+    double radius, sine, cosine;
+    orc_box_muller_parts(a, b, &radius, &sine, &cosine);
+    return (lane & 1) ? radius * sine : radius * cosine;
 }
 
 /* out[c] = orc_noise(seed, k, u, i0 + c) for c in [0, n): a convenience for statistical tests. */
 void orc_noise_fill(uint64_t seed, int64_t k, int64_t u, int64_t i0, int64_t n, double *out)
 {
+#pragma omp parallel for schedule(static)
     for (int64_t c = 0; c < n; ++c)
         out[c] = orc_noise(seed, k, u, i0 + c);
 }
@@ -222,11 +248,11 @@ int orc_local_step(const orc_config *c, int64_t rows, int64_t k0, int64_t n, con
                    real *theta, real *s1, real *s2, const real *grads,
                    int64_t t, int64_t n_state)
 {
-    const real eta = (real)orc_lr(c, t);
-    const real mu = (real)c->momentum;
-    const real b1 = (real)c->beta1, b2 = (real)c->beta2, eps = (real)c->eps;
-    const real bc1 = (real)(1.0 - pow(c->beta1, (double)(n_state + 1)));
-    const real bc2 = (real)(1.0 - pow(c->beta2, (double)(n_state + 1)));
+    const double eta = orc_lr(c, t);
+    const double mu = c->momentum;
+    const double b1 = c->beta1, b2 = c->beta2, eps = c->eps;
+    const double bc1 = 1.0 - pow(c->beta1, (double)(n_state + 1));
+    const double bc2 = 1.0 - pow(c->beta2, (double)(n_state + 1));
     real *g_row = (real *)malloc((size_t)(n > 0 ? n : 1) * sizeof(real));
     if (!g_row)
         return -1;
@@ -242,31 +268,31 @@ int orc_local_step(const orc_config *c, int64_t rows, int64_t k0, int64_t n, con
             else
                 g_row[col] = lambda[col] * (theta[e] - theta_star[col]) + (real)(c->noise_std * orc_noise(c->seed, k, t, i));
         }
-        real clip_coef = 1;
+        double clip_coef = 1.0;
         if (c->clip_norm > 0.0) {
             double sum_sq = 0.0;
             for (int64_t col = 0; col < n; ++col)
                 sum_sq += (double)g_row[col] * (double)g_row[col];
             double coef = c->clip_norm / (sqrt(sum_sq) + 1e-6);
-            clip_coef = (real)(coef < 1.0 ? coef : 1.0);
+            clip_coef = coef < 1.0 ? coef : 1.0;
         }
         /* OPT (Eq. 1) */
 #pragma omp parallel for schedule(static)
         for (int64_t col = 0; col < n; ++col) {
             const int64_t e = r * n + col;
-            const real wd = (real)(c->weight_decay * (c->wd_scale ? c->wd_scale[col] : 1.0));
-            real g = clip_coef * g_row[col];
+            const double wd = c->weight_decay * (c->wd_scale ? c->wd_scale[col] : 1.0);
+            double g = clip_coef * (double)g_row[col];
             if (c->opt == ORC_OPT_SGDM) {
-                g = g + wd * theta[e];
-                s1[e] = mu * s1[e] + g;
-                theta[e] = theta[e] - eta * s1[e];
+                g = g + wd * (double)theta[e];
+                s1[e] = (real)(mu * (double)s1[e] + g);
+                theta[e] = (real)((double)theta[e] - eta * (double)s1[e]);
             } else {
-                theta[e] = theta[e] * ((real)1 - eta * wd);
-                s1[e] = b1 * s1[e] + ((real)1 - b1) * g;
-                s2[e] = b2 * s2[e] + ((real)1 - b2) * g * g;
-                real m_hat = s1[e] / bc1;
-                real denom = (real)sqrt((double)s2[e]) / (real)sqrt((double)bc2) + eps;
-                theta[e] = theta[e] - eta * m_hat / denom;
+                double decayed = (double)theta[e] * (1.0 - eta * wd);
+                s1[e] = (real)(b1 * (double)s1[e] + (1.0 - b1) * g);
+                s2[e] = (real)(b2 * (double)s2[e] + (1.0 - b2) * g * g);
+                double m_hat = (double)s1[e] / bc1;
+                double denom = sqrt((double)s2[e]) / sqrt(bc2) + eps;
+                theta[e] = (real)(decayed - eta * m_hat / denom);
             }
         }
     }
@@ -290,14 +316,15 @@ int orc_parallel_step(const orc_config *c, int64_t K, int64_t n, const int64_t *
         return -1;
     for (int64_t col = 0; col < n; ++col) {
         const int64_t i = idx ? idx[col] : col;
-        real sum = 0;
+        double sum = 0.0;
         for (int64_t k = 0; k < K; ++k) {
             if (grads)
-                sum += grads[k * n + col];
+                sum += (double)grads[k * n + col];
             else
-                sum += lambda[col] * (theta[col] - theta_star[col]) + (real)(c->noise_std * orc_noise(c->seed, k, t, i));
+                sum += (double)lambda[col] * ((double)theta[col] - (double)theta_star[col])
+                       + c->noise_std * orc_noise(c->seed, k, t, i);
         }
-        g_mean[col] = sum / (real)K;
+        g_mean[col] = (real)(sum / (double)K);
     }
     /* clipping, when on, acts on the averaged gradient, as for the paper's parallel AdamW baseline */
     int rc = orc_local_step(c, 1, 0, n, idx, lambda, theta_star, theta, s1, s2, g_mean, t, n_state);
@@ -311,10 +338,10 @@ static void mean_rows(int64_t rows, int64_t n, real *x)
 {
 #pragma omp parallel for schedule(static)
     for (int64_t col = 0; col < n; ++col) {
-        real sum = 0;
+        double sum = 0.0;
         for (int64_t r = 0; r < rows; ++r)
-            sum += x[r * n + col];
-        real mean = sum / (real)rows;
+            sum += (double)x[r * n + col];
+        real mean = (real)(sum / (double)rows);
         for (int64_t r = 0; r < rows; ++r)
             x[r * n + col] = mean;
     }

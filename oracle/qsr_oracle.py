@@ -1,8 +1,8 @@
 """ctypes front end of the CPU oracle (qsr_oracle.c)  --  TEST INFRASTRUCTURE ONLY.
 
 Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this module.
-It compiles the C file with gcc on first use (binary64 build, and a binary32 "mirror" build used
-only to size rounding error) and marshals numpy arrays; it contains no arithmetic of its own
+It compiles the C file with gcc on first use (binary64 build, and a "mirror" build with binary32
+storage used only to size rounding error) and marshals numpy arrays; it contains no arithmetic of its own
 and imports nothing from the CUDA package.
 """
 from __future__ import annotations
@@ -71,6 +71,8 @@ def _lib(mirror: bool = False):
             lib.orc_noise.argtypes = [C.c_uint64, C.c_int64, C.c_int64, C.c_int64]
             lib.orc_noise_fill.restype = None
             lib.orc_noise_fill.argtypes = [C.c_uint64, C.c_int64, C.c_int64, C.c_int64, C.c_int64, p]
+            lib.orc_box_muller_parts_fill.restype = None
+            lib.orc_box_muller_parts_fill.argtypes = [p, p, C.c_int64, p, p, p]
             lib.orc_local_step.restype = C.c_int
             lib.orc_local_step.argtypes = [cfg, C.c_int64, C.c_int64, C.c_int64, p, p, p, p, p, p, p, C.c_int64, C.c_int64]
             lib.orc_parallel_step.restype = C.c_int
@@ -140,6 +142,16 @@ def noise_fill(seed: int, k: int, u: int, i0: int, n: int) -> np.ndarray:
     out = np.empty(int(n), np.float64)
     _lib().orc_noise_fill(C.c_uint64(seed), int(k), int(u), int(i0), int(n), _ptr(out))
     return out
+
+
+def box_muller_parts(a, b) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """(radius, sine, cosine) of the Box-Muller transform for arrays of 23-bit fields a (radius) and b (angle)."""
+    a = np.ascontiguousarray(a, np.uint32)
+    b = np.ascontiguousarray(b, np.uint32)
+    assert a.shape == b.shape and a.ndim == 1
+    radius, sine, cosine = (np.empty(a.size, np.float64) for _ in range(3))
+    _lib().orc_box_muller_parts_fill(_ptr(a), _ptr(b), a.size, _ptr(radius), _ptr(sine), _ptr(cosine))
+    return radius, sine, cosine
 
 
 class State:

@@ -28,7 +28,7 @@ QSR_STATIC_SCRATCH_FLOATS = 1 << 20
 EXPORTS = ("qsr_config_check", "qsr_row_stride_hint", "qsr_config_learning_rate", "qsr_config_round_length", "qsr_config_schedule",
            "qsr_workspace_bytes", "qsr_init", "qsr_destroy", "qsr_round_length", "qsr_set_tensor_table", "qsr_clip_workspace_floats", "qsr_set_grad_clip", "qsr_set_params", "qsr_local_step",
            "qsr_local_step_sync", "qsr_parallel_step", "qsr_sync", "qsr_sync_sum_floats", "qsr_sync_partial", "qsr_local_step_partial", "qsr_sync_finish", "qsr_sync_static", "qsr_run", "qsr_launch_count",
-           "qsr_set_launch_shape", "qsr_set_graph_replay", "qsr_train_host", "qsr_strerror")
+           "qsr_set_launch_shape", "qsr_set_graph_replay", "qsr_train_host", "qsr_debug_box_muller", "qsr_strerror")
 
 
 class QsrConfig(C.Structure):
@@ -89,6 +89,7 @@ def lib():
             "qsr_set_launch_shape": (C.c_int, [vp, i32, i32, i32]),
             "qsr_set_graph_replay": (C.c_int, [vp, i32]),
             "qsr_train_host": (C.c_int, [cfg, vp, vp, vp, vp, vp, i64, i64, vp, vp, vp, i64, C.POINTER(i64), C.POINTER(i64)]),
+            "qsr_debug_box_muller": (C.c_int, [vp, i64, vp, vp, vp, vp]),
             "qsr_strerror": (C.c_char_p, [C.c_int]),
         }
         for name in EXPORTS:
@@ -280,3 +281,10 @@ def qsr_train_host(cfg: QsrConfig, theta0: np.ndarray, lam: np.ndarray, theta_st
                                 _dptr(workspace), nbytes, t_end, C.c_void_p(stream),
                                 st.ctypes.data, H.ctypes.data, cap, C.byref(n), C.byref(launches)), "qsr_train_host")
     return st[:n.value].copy(), H[:n.value].copy(), int(launches.value)
+
+
+def qsr_debug_box_muller(words, radius, sine, cosine, stream: int = 0) -> None:
+    """Test hook: Box-Muller radius / sine / cosine of each uint32 generator word (CUDA tensors; words as int32 bits)."""
+    n = int(words.numel())
+    _check(lib().qsr_debug_box_muller(_dptr(words), n, _dptr(radius), _dptr(sine), _dptr(cosine), C.c_void_p(stream)),
+           "qsr_debug_box_muller")

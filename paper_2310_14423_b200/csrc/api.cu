@@ -27,6 +27,7 @@ struct qsr_ctx {
     float *theta, *s1, *s2;
     const float *lambda, *theta_star;
     cudaStream_t stream;
+    int device;               // ordinal of the device that was current at qsr_init
     qsr::LaunchShape shape;
     int64_t t_state_origin;
     int64_t launches;
@@ -226,6 +227,7 @@ int qsr_init(qsr_ctx **out, const qsr_config *cfg, float *params, float *state1,
     x->theta = params; x->s1 = state1; x->s2 = cfg->opt == QSR_OPT_ADAMW ? state2 : nullptr;
     x->lambda = lambda; x->theta_star = theta_star;
     x->stream = static_cast<cudaStream_t>(cuda_stream);
+    x->device = dev;
     x->shape = qsr::LaunchShape();
     if (cfg->opt == QSR_OPT_SGDM) x->shape.step_threads = 128;
     // Slabs that stay resident in L2 between steps are served with far lower latency than HBM: a 4-row ring in
@@ -287,12 +289,17 @@ int qsr_local_step(qsr_ctx *ctx, int64_t t, const float *grads)
 int qsr_set_tensor_table(qsr_ctx *ctx, int32_t n_tensors, const int64_t *tensor_end_dev, const float *wd_scale_dev)
 {
     if (!ctx || n_tensors < 0) return QSR_EINVAL;
+    if (n_tensors > 0) {
+        if (!tensor_end_dev || !wd_scale_dev) return QSR_EINVAL;
+        if ((reinterpret_cast<uintptr_t>(tensor_end_dev) & 7u) || (reinterpret_cast<uintptr_t>(wd_scale_dev) & 3u)) return QSR_EALIGN;
+    }
+    // A table switches the step to the kernel instance that looks the factors up; cached graph chains were built
+    // around the other instance and would go on replaying it, so they are discarded whenever the choice changes.
+    if ((ctx->n_tensors > 0) != (n_tensors > 0)) drop_graphs(*ctx);
     if (n_tensors == 0) {
         ctx->n_tensors = 0; ctx->tensor_end = nullptr; ctx->wd_scale = nullptr;
         return QSR_OK;
     }
-    if (!tensor_end_dev || !wd_scale_dev) return QSR_EINVAL;
-    if ((reinterpret_cast<uintptr_t>(tensor_end_dev) & 7u) || (reinterpret_cast<uintptr_t>(wd_scale_dev) & 3u)) return QSR_EALIGN;
     ctx->n_tensors = n_tensors; ctx->tensor_end = tensor_end_dev; ctx->wd_scale = wd_scale_dev;
     return QSR_OK;
 }
@@ -422,11 +429,23 @@ int qsr_sync_static(qsr_ctx *ctx, int64_t t_next)
     if (t_next < 0 || t_next > ctx->cfg.T) return QSR_ERANGE;
     const qsr::SyncParams p = sync_params(*ctx);
     if (int64_t(p.n_mean) * p.P4 > int64_t(QSR_STATIC_SCRATCH_FLOATS)) return QSR_ERANGE;   // nothing was launched
-    const int err = qsr::launch_sync_static(p, ctx->shape, ctx->stream);
-    if (err != 0) return err == -1 ? QSR_ERANGE : QSR_ECUDA;
+    const int err = qsr::launch_sync_static(p, ctx->shape, ctx->device, ctx->stream);
+    if (err != 0) return err == -1 ? QSR_ERANGE : (err == -2 ? QSR_ESTATE : QSR_ECUDA);
     ctx->launches += 2;
     if (ctx->cfg.state_sync == QSR_STATE_RESET) ctx->t_state_origin = t_next;
     return QSR_OK;
+}
+
+int qsr_debug_box_muller(const uint32_t *words_dev, int64_t n, float *radius_dev, float *sin_dev, float *cos_dev,
+                         void *cuda_stream)
+{
+    if (n < 0) return QSR_EINVAL;
+    if (n == 0) return QSR_OK;
+    if (!words_dev || !radius_dev || !sin_dev || !cos_dev) return QSR_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(words_dev) | reinterpret_cast<uintptr_t>(radius_dev) |
+         reinterpret_cast<uintptr_t>(sin_dev) | reinterpret_cast<uintptr_t>(cos_dev)) & 3u)
+        return QSR_EALIGN;
+    return cuda_rc(qsr::launch_box_muller_parts(words_dev, n, radius_dev, sin_dev, cos_dev, cuda_stream));
 }
 
 int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
@@ -512,6 +531,8 @@ int qsr_train_host(const qsr_config *cfg, const float *theta0_host, const float 
                    void *workspace_dev, int64_t workspace_bytes, int64_t t_end, void *cuda_stream,
                    int64_t *round_start, int64_t *round_len, int64_t cap, int64_t *n_rounds, int64_t *launches)
 {
+    if (launches) *launches = 0;
+    if (n_rounds) *n_rounds = 0;
     if (!cfg || !theta0_host || !lambda_host || !theta_star_host || !theta_out_host || !workspace_dev) return QSR_EINVAL;
     qsr_config c = *cfg;
     c.row_stride = qsr::row_stride_hint(c.P);
@@ -529,14 +550,18 @@ int qsr_train_host(const qsr_config *cfg, const float *theta0_host, const float 
     float *lambda = vec, *theta_star = vec + c.row_stride, *theta0 = vec + 2 * c.row_stride;
     const size_t row_bytes = size_t(c.P) * sizeof(float);
 
-    if (cudaMemcpyAsync(lambda, lambda_host, row_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return QSR_ECUDA;
-    if (cudaMemcpyAsync(theta_star, theta_star_host, row_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return QSR_ECUDA;
-    if (cudaMemcpyAsync(theta0, theta0_host, row_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return QSR_ECUDA;
-    if (cudaMemsetAsync(s1, 0, size_t(n_state_slabs(c)) * slab * sizeof(float), st) != cudaSuccess) return QSR_ECUDA;
-
+    // Every check that can fail on the host comes before the first copy is enqueued (the context only records
+    // pointers); from here on, whatever happens, the call waits for the stream before it returns, so the caller's
+    // host buffers are never still in use by a copy when it gets them back.
     qsr_ctx *x = nullptr;
     if (int rc = qsr_init(&x, &c, theta, s1, s2, lambda, theta_star, cuda_stream)) return rc;
-    int rc = qsr_set_params(x, theta0);
+    int rc = QSR_OK;
+    if (cudaMemcpyAsync(lambda, lambda_host, row_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(theta_star, theta_star_host, row_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(theta0, theta0_host, row_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemsetAsync(s1, 0, size_t(n_state_slabs(c)) * slab * sizeof(float), st) != cudaSuccess)
+        rc = QSR_ECUDA;
+    if (rc == QSR_OK) rc = qsr_set_params(x, theta0);
     if (rc == QSR_OK) rc = qsr_run(x, 0, t_end, round_start, round_len, cap, n_rounds);
     if (rc == QSR_OK && cudaMemcpyAsync(theta_out_host, theta, row_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         rc = QSR_ECUDA;

@@ -90,8 +90,11 @@ int launch_broadcast(float *theta, const float *theta0, int64_t P, int64_t strid
 // Gradient clipping: grid of the norm pass and the two passes that leave the factors at ws + clip_grid(...) * rows.
 int clip_grid(int64_t P);
 int launch_clip_coef(const StepParams &p, bool parallel, double max_norm, float *ws, const LaunchShape &shape, void *stream);
-// Both phases through the library's own static scratch; -1 if the sums exceed QSR_STATIC_SCRATCH_FLOATS.
-int launch_sync_static(const SyncParams &p, const LaunchShape &shape, void *stream);
+// Test hook: radius, sine and cosine of the Box-Muller transform for n generator words (all device arrays).
+int launch_box_muller_parts(const uint32_t *words, int64_t n, float *radius, float *sine, float *cosine, void *stream);
+// Both phases through the library's own static scratch; -1 if the sums exceed QSR_STATIC_SCRATCH_FLOATS, -2 if
+// `device` (the context's) is not the current device.
+int launch_sync_static(const SyncParams &p, const LaunchShape &shape, int device, void *stream);
 
 }  // namespace qsr
 #endif

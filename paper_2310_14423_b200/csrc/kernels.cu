@@ -8,6 +8,7 @@
 // per thread in flight through a cp.async ring in shared memory to cover HBM latency.
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdint>
 
 #include "internal.h"
@@ -571,6 +572,25 @@ __global__ void __launch_bounds__(512) broadcast_kernel(float *theta, const floa
     }
 }
 
+// ---------------------------------------------------------------------------------------------- test hook
+//
+// The two halves of the Box-Muller transform for a list of generator words, through the very device functions the
+// step kernels inline (neg2_log_unit, sqrt_fast, sincos_turn_bits): word w gives the radius sqrt(-2 ln u) for
+// u = (w >> 9 + 1/2) / 2^23 and the sine / cosine of the angle 2 pi u.  The grid of inputs has only 2^23 points, so a
+// test can walk all of it and bound the error of each part against binary64.
+__global__ void box_muller_parts_kernel(const uint32_t *words, int64_t n, float *radius, float *sine, float *cosine)
+{
+    const int64_t grid_stride = int64_t(gridDim.x) * blockDim.x;
+    for (int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += grid_stride) {
+        const uint32_t w = words[i];
+        float s, c;
+        sincos_turn_bits(w, s, c);
+        radius[i] = sqrt_fast(neg2_log_unit(w));
+        sine[i] = s;
+        cosine[i] = c;
+    }
+}
+
 // One thread per 16-byte column.  2^31 - 1 blocks of at least 64 threads cover rows of 2^39 floats, beyond any device
 // memory, so the kernels that rely on full coverage (local_step_kernel) never meet a capped grid.
 unsigned grid_for(int64_t P, int threads)
@@ -736,6 +756,15 @@ int launch_broadcast(float *theta, const float *theta0, int64_t P, int64_t strid
     return int(cudaGetLastError());
 }
 
+int launch_box_muller_parts(const uint32_t *words, int64_t n, float *radius, float *sine, float *cosine, void *stream)
+{
+    int64_t blocks = (n + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks < 1) blocks = 1;
+    box_muller_parts_kernel<<<unsigned(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(words, n, radius, sine, cosine);
+    return int(cudaGetLastError());
+}
+
 }  // namespace qsr
 
 // ---------------------------------------------------------------------------------------------- static scratch
@@ -750,24 +779,28 @@ namespace qsr {
 
 namespace {
 constexpr int kMaxDevices = 64;
-float *g_scratch_addr[kMaxDevices] = {};   // device address of g_sync_scratch, per device ordinal (0 = not yet asked)
+// Device address of g_sync_scratch per device ordinal (null = not yet asked).  Atomic, so that contexts on different
+// host threads may make their first call at the same time: both look the same address up and store the same value.
+std::atomic<float *> g_scratch_addr[kMaxDevices];
 }  // namespace
 
 // The two phases (row sums into the static array, then rows <- sums / K) enqueued back to back on `stream`.
-// Returns 0, a cudaError_t, or -1 when the sums do not fit.  The first call on a device looks the array's device
-// address up; no memory is allocated or freed here.
-int launch_sync_static(const SyncParams &p_in, const LaunchShape &shape, void *stream)
+// `device` is the ordinal the context was created on; it must be the current one, because the array's address is
+// looked up for the current device.  Returns 0, a cudaError_t, -1 when the sums do not fit, -2 when another device
+// is current.  The first call on a device looks the array's device address up; no memory is allocated or freed here.
+int launch_sync_static(const SyncParams &p_in, const LaunchShape &shape, int device, void *stream)
 {
     if (int64_t(p_in.n_mean) * p_in.P4 > int64_t(QSR_STATIC_SCRATCH_FLOATS)) return -1;
     int dev = -1;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return int(err);
+    if (dev != device) return -2;
     if (dev < 0 || dev >= kMaxDevices) return int(cudaErrorInvalidDevice);
-    float *scratch = g_scratch_addr[dev];
+    float *scratch = g_scratch_addr[dev].load(std::memory_order_acquire);
     if (!scratch) {
         err = cudaGetSymbolAddress(reinterpret_cast<void **>(&scratch), g_sync_scratch);
         if (err != cudaSuccess) return int(err);
-        g_scratch_addr[dev] = scratch;
+        g_scratch_addr[dev].store(scratch, std::memory_order_release);
     }
     // Every float the second phase reads is written by the first phase of the same call, so nothing left in the
     // array by an earlier call can leak into this one and nothing has to be cleared.

@@ -105,3 +105,33 @@ def test_argument_errors():
         assert e.value.status == B.QSR_ERANGE
     ctx.qsr_set_graph_replay(0)
     ctx.close()
+
+
+def test_tensor_table_set_between_replayed_runs():
+    """A per-tensor weight-decay table set (or cleared) between two replayed runs switches the step to another kernel
+    instance; the cached chains must not go on replaying the old one.  Replay on, a stretch of rounds, a table that
+    switches weight decay off for one tensor, the rest of the run, the table cleared, and again -- against a context
+    that launches everything directly."""
+    w = W.tiny_workload(W.OPT_ADAMW, K=3, P=4096, T=300, weight_decay=0.1)
+    lam, ths, lam_d, ths_d = G.device_inputs(w)
+    ends = torch.tensor([1024, 2048, 4096], dtype=torch.int64, device="cuda")
+    scales = torch.tensor([1.0, 0.0, 2.0], device="cuda")
+    runs = []
+    for graph_steps in (0, 16):
+        S = G.Slabs(w)
+        ctx = G.make_context(w, S, lam_d, ths_d)
+        ctx.qsr_set_graph_replay(graph_steps)
+        st_a, H_a = ctx.qsr_run(0, 100)
+        t1 = int(st_a[-1] + H_a[-1])
+        ctx.qsr_set_tensor_table(ends, scales)
+        st_b, H_b = ctx.qsr_run(t1, 200)
+        t2 = int(st_b[-1] + H_b[-1])
+        ctx.qsr_set_tensor_table(None, None)
+        ctx.qsr_run(t2, w.T)
+        torch.cuda.synchronize()
+        ctx.close()
+        runs.append(S)
+    assert _same(runs[0], runs[1])
+    # and the table did act in the middle stretch: a run without it ends elsewhere
+    _, _, plain, _, _, _ = _run(w, 0)
+    assert not torch.equal(plain.theta, runs[0].theta)

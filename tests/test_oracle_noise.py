@@ -47,23 +47,37 @@ def test_pair_lies_on_one_circle():
     assert abs(r2.mean() - 2.0) < 4 * 2.0 / math.sqrt(r2.size)
 
 
+N_DRAWS = 1 << 24          # 1.7e7 normals per statistical test
+
+
 def test_moments_and_uniformity():
-    n = 1 << 21
+    n = N_DRAWS
     z = O.noise_fill(SEED, 0, 0, 0, n)
     se = 1 / math.sqrt(n)
     assert abs(z.mean()) < 4 * se
-    assert abs(z.var() - 1) < 4 * math.sqrt(2) * se
+    assert abs(z.var() - 1) < 4 * math.sqrt(2) * se          # far inside the 1 % band
     assert abs((z ** 3).mean()) < 4 * math.sqrt(15) * se
     assert abs((z ** 4).mean() - 3) < 4 * math.sqrt(96) * se
     assert np.abs(z).max() < math.sqrt(2 * 24 * math.log(2)) + 1e-9
     for lane in range(4):
-        p = stats.kstest(z[lane::4][:200000], "norm").pvalue
+        p = stats.kstest(z[lane::4], "norm").pvalue
         assert p > 1e-4, (lane, p)
+    # the two uniforms behind every pair, recovered from the normals: u1 = exp(-(z0^2 + z1^2)/2), u2 = angle / 2 pi
+    z0, z1 = z[0::2], z[1::2]
+    u1 = np.exp(-0.5 * (z0 * z0 + z1 * z1))
+    u2 = np.mod(np.arctan2(z1, z0) / (2 * math.pi), 1.0)
+    for name, u in (("u1", u1), ("u2", u2)):
+        p = stats.kstest(u, "uniform").pvalue
+        assert p > 1e-4, (name, p)
+        # they sit on the grid (a + 1/2) / 2^23
+        a = u[:100000] * 2 ** 23 - 0.5
+        assert np.abs(a - np.round(a)).max() < 1e-3, name
+    assert abs(np.corrcoef(u1, u2)[0, 1]) < 4.5 / math.sqrt(u1.size)
 
 
 def test_independence_across_workers_steps_and_neighbours():
-    n = 1 << 19
-    bound = 4.5 / math.sqrt(n)
+    n = N_DRAWS
+    bound = 4 / math.sqrt(n)
     base = O.noise_fill(SEED, 0, 0, 0, n)
     others = {
         "worker": O.noise_fill(SEED, 1, 0, 0, n),
@@ -77,6 +91,58 @@ def test_independence_across_workers_steps_and_neighbours():
         assert abs(np.corrcoef(base[:-lag], base[lag:])[0, 1]) < bound, lag
     # within a pair the two branches are uncorrelated, also in their squares
     assert abs(np.corrcoef(base[0::2] ** 2, base[1::2] ** 2)[0, 1]) < 2 * bound
+
+
+def test_box_muller_parts_against_40_digit_arithmetic():
+    """radius = sqrt(-2 ln u1), sin / cos(2 pi u2) on the 23-bit grid: the ends of the grid, the quadrant borders and
+    seeded random fields, against mpmath at 40 digits."""
+    import mpmath
+    mpmath.mp.dps = 40
+    rng = np.random.default_rng(7)
+    n_grid = 1 << 23
+    edge = [0, 1, 2, n_grid - 1, n_grid - 2, n_grid // 2, n_grid // 2 - 1, n_grid // 4, n_grid // 4 - 1,
+            3 * n_grid // 4, 3 * n_grid // 4 - 1, n_grid // 8, 12345]
+    a = np.array(edge + rng.integers(0, n_grid, 1500).tolist(), np.uint32)
+    b = np.array(edge[::-1] + rng.integers(0, n_grid, 1500).tolist(), np.uint32)
+    radius, sine, cosine = O.box_muller_parts(a, b)
+    for i in range(a.size):
+        u1 = (mpmath.mpf(int(a[i])) + mpmath.mpf(1) / 2) / n_grid
+        u2 = (mpmath.mpf(int(b[i])) + mpmath.mpf(1) / 2) / n_grid
+        r = mpmath.sqrt(-2 * mpmath.log(u1))
+        assert abs(mpmath.mpf(float(radius[i])) - r) <= 4e-16 * r
+        # the product 2 pi u2 is rounded to binary64 before the sine: an argument error of up to 4e-16 near 2 pi
+        assert abs(mpmath.mpf(float(sine[i])) - mpmath.sin(2 * mpmath.pi * u2)) <= 1e-15
+        assert abs(mpmath.mpf(float(cosine[i])) - mpmath.cos(2 * mpmath.pi * u2)) <= 1e-15
+
+
+def test_box_muller_parts_over_the_whole_grid():
+    """All 2^23 fields: the angle grid is symmetric, so sine and cosine average to zero; sin^2 + cos^2 = 1; the mean of
+    radius^2 = -2 ln u1 over the midpoint grid is 2 (the integral) up to the midpoint rule's error at the singularity."""
+    n_grid = 1 << 23
+    f = np.arange(n_grid, dtype=np.uint32)
+    radius, sine, cosine = O.box_muller_parts(f, f)
+    assert abs(sine.mean()) < 1e-13 and abs(cosine.mean()) < 1e-13
+    assert np.abs(sine * sine + cosine * cosine - 1).max() < 1e-15
+    assert np.array_equal(np.sign(sine[:n_grid // 2]), np.ones(n_grid // 2))          # first half turn: sine > 0
+    assert np.abs(sine + sine[::-1]).max() < 1e-15 and np.abs(cosine - cosine[::-1]).max() < 1e-15
+    assert np.all(np.diff(radius) < 0)                                                # radius falls as u1 grows
+    # midpoint rule for the integral of -2 ln u over (0,1): error ~ ln(2)/N from the first cell
+    assert abs((radius * radius).mean() - 2.0) < 2.0 / n_grid
+    assert radius[0] == math.sqrt(2 * 24 * math.log(2))
+
+
+def test_noise_is_radius_times_branch():
+    """orc_noise for coordinate i equals the parts' radius times cosine (even lane) or sine (odd lane), bit for bit."""
+    for (k, u, i0) in [(0, 0, 0), (7, 4242, 4 * 10 ** 6)]:
+        z = O.noise_fill(SEED, k, u, i0, 64)
+        for c in range(64):
+            i = i0 + c
+            j = i >> 2
+            r = O.philox4x32_10([j & 0xFFFFFFFF, j >> 32, u, k], [SEED & 0xFFFFFFFF, SEED >> 32])
+            lane = i & 3
+            a, b = int(r[2 * (lane >> 1)]) >> 9, int(r[2 * (lane >> 1) + 1]) >> 9
+            radius, sine, cosine = O.box_muller_parts([a], [b])
+            assert z[c] == radius[0] * (sine[0] if lane & 1 else cosine[0])
 
 
 def test_noise_is_a_pure_function_of_its_four_integers():

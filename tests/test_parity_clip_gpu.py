@@ -26,11 +26,9 @@ def _clip_context(w, S, lam_d, ths_d):
 def test_clipped_local_runs(opt, K, P):
     # the threshold sits inside the range of gradient norms of the run, so some steps clip and some do not
     clip = {3: 0.02, 1001: 3.0, 40002: 20.0, 300000: 55.0}[P]
-    # Adam's first steps divide by the root of a second moment that has seen only a few gradients: about one coordinate
-    # in 1e5 (here: coordinate 53772, with or without clipping, also in the oracle's own binary32 build) reacts to fp32
-    # rounding there with an error of a few 1e-5 that the later steps contract away (2.5e-4 after 30 steps, 2.4e-5
-    # after 120, 1.5e-6 after 480).  These runs start at full learning rate, so the largest case runs 480 steps.
-    w = W.tiny_workload(opt, K=K, P=P, T=480 if P > 100000 else 30, clip_norm=clip)
+    # the largest AdamW case starts at the full learning rate, where one coordinate in 1e5 is ill-conditioned for any
+    # fp32 gradient (see conditioning.py); assert_parity bounds it by the run's own sensitivity instead of avoiding it
+    w = W.tiny_workload(opt, K=K, P=P, T=30, clip_norm=clip)
     lam, ths, lam_d, ths_d = G.device_inputs(w)
     S = G.Slabs(w)
     ctx, ws = _clip_context(w, S, lam_d, ths_d)
@@ -40,7 +38,8 @@ def test_clipped_local_runs(opt, K, P):
     orc = G.oracle_on(w, lam, ths)
     ost, oH = orc.run()
     assert np.array_equal(st, ost) and np.array_equal(H, oH)
-    assert G.rel_err(S.theta[:, :P].cpu().numpy(), orc.theta) <= G.REL_TOL
+    G.assert_parity(S.theta[0, :P].cpu().numpy(), w, lam, ths, orc.theta[0])
+    assert bool((S.theta[:, :P] == S.theta[0, :P]).all())
     free = G.oracle_on(w.replace(clip_norm=0.0), lam, ths)
     free.run()
     assert G.rel_err(S.theta[0, :P].cpu().numpy(), free.theta[0]) > 1e-4   # clipping did change the run

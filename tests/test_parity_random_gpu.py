@@ -1,7 +1,9 @@
 """Seeded random configurations through the C ABI against the CPU oracle: worker counts, ragged sizes, padded row
 strides, launch shapes, every round-length rule, learning-rate schedule and state mode in combinations that the
-hand-picked cases of test_parity_gpu.py do not enumerate.  Bars as there: the round log bit-exact, parameters within
-REL_TOL on every coordinate."""
+hand-picked cases of test_parity_gpu.py do not enumerate -- AdamW started at full learning rate and AdamW whose
+moments are reset at every synchronization included.  Bars: the round log bit-exact; parameters within REL_TOL on every
+coordinate; a coordinate may miss it only by what the run's own conditioning explains (gpu_harness.assert_parity:
+the binary64 oracle, its gradients perturbed by one fp32 ulp, must move that coordinate as far)."""
 import numpy as np
 import pytest
 import torch
@@ -21,10 +23,8 @@ def _draw(case):
     opt = (W.OPT_SGDM, W.OPT_ADAMW)[int(rng.integers(2))]
     K = int(rng.choice([1, 2, 3, 4, 7, 8, 9, 16, 19, 33]))
     P = int(rng.choice([1, 6, 7, 255, 1000, 1025, 2047, 4100, 9999]))
-    # AdamW's first steps at full learning rate amplify fp32 rounding on a few coordinates (contracted away after a
-    # few hundred steps), so its short runs warm up from zero, as the run configurations do
-    T = int(rng.integers(30, 90)) if opt == W.OPT_SGDM else int(rng.integers(300, 420))
-    T_warmup = int(rng.integers(0, T // 3)) if opt == W.OPT_SGDM else int(rng.integers(40, 100))
+    T = int(rng.integers(30, 90)) if rng.integers(2) else int(rng.integers(300, 420))
+    T_warmup = int(rng.integers(0, T // 3))
     sched = str(rng.choice([W.SCHED_COSINE, W.SCHED_STEP_POW2, W.SCHED_LINEAR, W.SCHED_CONST, W.SCHED_HALVING,
                             W.SCHED_COSINE_HELD]))
     rule = str(rng.choice([W.RULE_QSR, W.RULE_QSR, W.RULE_CONST_H, W.RULE_POWER, W.RULE_POST_LOCAL, W.RULE_SWAP]))
@@ -35,11 +35,7 @@ def _draw(case):
               t_hold=int(rng.integers(T_warmup, T)), t_period=int(rng.integers(1, 12)),
               momentum=float(rng.choice([0.0, 0.5, 0.9])), weight_decay=float(rng.choice([0.0, 1e-4, 0.05])),
               noise_std=float(rng.choice([0.0, 0.05, 0.2])),
-              # resetting Adam's moments at every synchronization makes each round start with sign-like steps
-              # g / (|g| + eps), which are ill-conditioned near the optimum: RESET is drawn for SGD only here
-              # (test_state_modes covers AdamW with RESET on a well-conditioned case)
-              state_sync=str(rng.choice([W.STATE_KEEP, W.STATE_KEEP, W.STATE_AVERAGE,
-                                         W.STATE_RESET if opt == W.OPT_SGDM else W.STATE_KEEP])),
+              state_sync=str(rng.choice([W.STATE_KEEP, W.STATE_KEEP, W.STATE_AVERAGE, W.STATE_RESET])),
               noise_seed=int(rng.integers(1, 2 ** 62)))
     w = W.tiny_workload(opt, K=K, P=P, T=T, **kw)
     P4 = (P + 3) // 4 * 4
@@ -67,6 +63,5 @@ def test_random_configuration(case):
     assert int(st[-1] + H[-1]) == w.T
     theta = S.theta[:, :w.P].cpu().numpy()
     assert (theta == theta[0]).all()                    # the run ends with a synchronization
-    err = G.rel_err(theta[0], orc.theta[0])
-    assert err <= G.REL_TOL, (err, w, stride, shape)
+    G.assert_parity(theta[0], w, lam, ths, orc.theta[0], context=(w, stride, shape))
     assert S.guards_intact()
