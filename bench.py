@@ -20,6 +20,7 @@ a round's last step carries the averaging itself (one launch, no extra HBM traff
 from __future__ import annotations
 
 import argparse
+import datetime
 import hashlib
 import json
 import os
@@ -86,25 +87,49 @@ def step_source_hash():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle samples of one GPU every 200 ms while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+    """nvidia-smi clock / throttle samples of one GPU every 50 ms, each with its time stamp.  It is started before the
+    warm-up launches (the tool needs a few hundred ms to come up) and `stop(t0, t1)` keeps the samples taken between
+    the host times t0 and t1 that bracket the timed region, so that even a window of a tenth of a second carries
+    readings taken under its own load."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    PERIOD_MS = 50
 
     def __init__(self, gpu_id: str):
         self.gpu_id = gpu_id
         self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", gpu_id, f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                          "--format=csv,noheader,nounits", "-lms", str(self.PERIOD_MS)],
                                          stdout=self.tmp, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    @staticmethod
+    def parse(lines, t0=None, t1=None, slack_s=0.0):
+        """[(sm, sm_max, power, reasons)] of the samples stamped within [t0 - slack, t1 + slack] (all if t0 is None)."""
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        out = []
+        for line in lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                stamp = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                sm, smax, power = float(parts[1]), float(parts[2]), float(parts[3])
+            except ValueError:
+                continue
+            if t0 is not None and not (t0 - slack_s <= stamp <= t1 + slack_s):
+                continue
+            out.append((sm, smax, power, {n for n, v in zip(names, parts[5:9]) if v.lower().startswith("active")}))
+        return out
+
+    def stop(self, t0: float, t1: float):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "period_ms": self.PERIOD_MS}
         if self.proc is None:
             return out
+        time.sleep(2e-3 * self.PERIOD_MS)          # let the sample that covers the end of the region be written
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -113,37 +138,18 @@ class ClockSampler:
         self.tmp.flush()
         self.tmp.seek(0)
         lines = self.tmp.readlines()
-        late = not lines
-        if late:
-            # the timed region ended before the first 200 ms sample: take one reading now
-            try:
-                lines = subprocess.run(["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.FIELDS}",
-                                        "--format=csv,noheader,nounits"], capture_output=True, text=True,
-                                       timeout=20).stdout.splitlines()
-            except Exception:
-                lines = []
-        sm, smax, power, reasons = [], [], [], set()
-        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for line in lines:
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 8:
-                continue
-            try:
-                sm.append(float(parts[0]))
-                smax.append(float(parts[1]))
-                power.append(float(parts[2]))
-            except ValueError:
-                continue
-            for name, val in zip(names, parts[4:8]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
         self.tmp.close()
         os.unlink(self.tmp.name)
-        if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(smax)), reasons=sorted(reasons),
-                       samples=len(sm), power_w_median=float(np.median(power)))
-            if late:
-                out["note"] = "one reading taken right after the timed region, which was shorter than the sampling period"
+        rows = self.parse(lines, t0, t1)
+        if not rows:
+            # a region shorter than the sampling period can fall between two samples: take its nearest neighbours
+            rows = self.parse(lines, t0, t1, slack_s=1e-3 * self.PERIOD_MS)
+            if rows:
+                out["note"] = f"the timed region fell between two samples; these are the ones within {self.PERIOD_MS} ms of it"
+        if rows:
+            reasons = set().union(*[r[3] for r in rows])
+            out.update(sm_mhz=float(np.median([r[0] for r in rows])), sm_max_mhz=float(max(r[1] for r in rows)),
+                       reasons=sorted(reasons), samples=len(rows), power_w_median=float(np.median([r[2] for r in rows])))
         return out
 
 
@@ -210,52 +216,111 @@ def cpu_baseline(w, budget_s=12.0):
                       f"binary64, {dt:.1f} s"}
 
 
-def main():
-    args = parse_args()
-    if args.impl == "reference":
-        run_reference(args)
-        return
+class CudaBackend:
+    """Everything of the measurement that touches a device, a stream or the process group.  The timed loop, the rank
+    bookkeeping and the JSON line are written against this small surface, so that the CPU tests can run the whole
+    multi-rank flow over gloo with stand-ins for the device parts."""
+    name = "cuda"
 
+    def __init__(self, rank: int, local_rank: int, world: int):
+        import torch
+        self.torch = torch
+        self.rank, self.world = rank, world
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+        torch.cuda.set_device(local_rank)
+        self.local_rank = local_rank
+        self.dev = torch.device("cuda", local_rank)
+
+    def init_process_group(self):
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=self.dev)
+
+    def zeros(self, *shape):
+        return self.torch.zeros(*shape, device=self.dev)
+
+    def empty_bytes(self, n):
+        return self.torch.empty(n, dtype=self.torch.uint8, device=self.dev)
+
+    def pinned(self, array=None, n=None):
+        t = self.torch.from_numpy(array) if array is not None else self.torch.zeros(n, dtype=self.torch.float32)
+        return t.pin_memory()
+
+    def stream(self) -> int:
+        return self.torch.cuda.current_stream().cuda_stream
+
+    def context(self, cfg, theta, s1, s2, lam, ths):
+        from paper_2310_14423_b200 import binding as B
+        return B.Context(cfg, theta, s1, s2, lam, ths, stream=self.stream())
+
+    def train_host(self, cfg, theta0, lam, ths, out, ws, t_end):
+        from paper_2310_14423_b200 import binding as B
+        return B.qsr_train_host(cfg, theta0, lam, ths, out, ws, t_end=t_end, stream=self.stream())
+
+    def event(self):
+        return self.torch.cuda.Event(enable_timing=True)
+
+    def synchronize(self):
+        self.torch.cuda.synchronize()
+
+    def release_cached_memory(self):
+        self.torch.cuda.empty_cache()
+
+    def clock_sampler(self):
+        uuid = str(self.torch.cuda.get_device_properties(self.local_rank).uuid)
+        return ClockSampler("GPU-" + uuid.replace("GPU-", ""))
+
+
+def rank_layout(base, world: int, rank: int):
+    """(workers held by this rank, workers in the whole job, global index of this rank's first worker): weak scaling,
+    every GPU holds the configuration's K workers, rank r the workers r*K .. r*K + K - 1."""
+    return base.K, base.K * world, rank * base.K
+
+
+def max_over_ranks(ms: float, backend) -> float:
+    """A time measured on each rank's own device -> the slowest rank's (the job is as fast as that)."""
+    if backend.world == 1:
+        return float(ms)
     import torch
+    import torch.distributed as dist
+    t = backend.zeros(1).double()
+    t += ms
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def run_ours(args, backend):
+    """The measurement on this rank.  Returns the result (a dict) on rank 0 and None elsewhere."""
     import torch.distributed as dist
     from paper_2310_14423_b200 import binding as B
     from paper_2310_14423_b200 import sharded
     from paper_2310_14423_b200 import workloads as W
 
     B.lib()  # fail loudly if the CUDA library is missing
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
+    world, rank = backend.world, backend.rank
     if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+        backend.init_process_group()
 
     base = W.workload(args.workload)
-    K_local = base.K                          # weak scaling: every GPU holds the configuration's K workers
-    K_total = K_local * world
-    w = base.replace(worker_offset=rank * K_local)
+    K_local, K_total, worker_offset = rank_layout(base, world, rank)
+    w = base.replace(worker_offset=worker_offset)
     steps, warmup = args.steps, max(args.warmup, 3)
     if steps > w.T:
         raise SystemExit(f"--steps must be <= {w.T}")
 
     lam_h, ths_h = W.draw_inputs(w.P, w.data_seed)
     P4 = (w.P + 3) // 4 * 4
-    lam = torch.zeros(P4, device=dev)
-    ths = torch.zeros(P4, device=dev)
-    lam[:w.P].copy_(torch.from_numpy(lam_h))
-    ths[:w.P].copy_(torch.from_numpy(ths_h))
+    lam = backend.zeros(P4)
+    ths = backend.zeros(P4)
+    lam[:w.P].copy_(backend.torch.from_numpy(lam_h))
+    ths[:w.P].copy_(backend.torch.from_numpy(ths_h))
     # rows on large power-of-two boundaries (see include/qsr.h) unless asked to pack them
     stride = P4 if args.packed_rows else B.qsr_row_stride_hint(w.P)
-    theta = torch.zeros(K_local, stride, device=dev)
-    s1 = torch.zeros(K_local, stride, device=dev)
-    s2 = torch.zeros(K_local, stride, device=dev) if w.opt == W.OPT_ADAMW else None
-    stream = torch.cuda.current_stream().cuda_stream
+    theta = backend.zeros(K_local, stride)
+    s1 = backend.zeros(K_local, stride)
+    s2 = backend.zeros(K_local, stride) if w.opt == W.OPT_ADAMW else None
     cfg = B.make_config(w, K=K_local, row_stride=stride)
     sharded_path = world > 1 or args.sharded_path      # rounds end with partial sums + all-reduce + finish
-    sums = torch.zeros(3 * P4, device=dev) if sharded_path else None
 
     def all_reduce(buf):
         if world > 1:
@@ -266,67 +331,58 @@ def main():
         s1.zero_()
         if s2 is not None:
             s2.zero_()
-        return B.Context(cfg, theta, s1, s2, lam, ths, stream=stream)
+        return backend.context(cfg, theta, s1, s2, lam, ths)
 
-    def do_sync(ctx, t_next):
+    def exchange_for(ctx):
         if not sharded_path:
-            ctx.qsr_sync(t_next)
-        else:
-            ctx.qsr_sync_partial(sums)
-            all_reduce(sums[:ctx.qsr_sync_sum_floats()])
-            ctx.qsr_sync_finish(sums, K_total, t_next)
+            return None
+        return sharded.Exchange(backend.zeros(ctx.qsr_sync_sum_floats()), K_total, all_reduce)
+
+    # ---- clocks are sampled from before the warm-up on; the samples inside the timed region are kept
+    sampler = backend.clock_sampler() if rank == 0 else None
 
     # ---- warm-up: a few steps and one synchronization, then start again from zero
     ctx = fresh_context()
+    ex = exchange_for(ctx)
     for t in range(warmup):
         ctx.qsr_local_step(t)
-    do_sync(ctx, warmup)
-    torch.cuda.synchronize()
+    if ex is None:
+        ctx.qsr_sync(warmup)
+    else:
+        ctx.qsr_sync_partial(ex.sums)
+        ex.all_reduce(ex.sums)
+        ctx.qsr_sync_finish(ex.sums, K_total, warmup)
+    backend.synchronize()
     ctx.close()
     ctx = fresh_context()
 
-    # ---- timed region: global steps [0, steps) with the syncs the schedule places in it
-    starts, H = B.qsr_config_schedule(cfg)
-    ends = set((starts + H).tolist())
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * steps + 2)]
+    # ---- timed region: global steps [0, steps) with the round ends the schedule places in it, through the same
+    #      loop (sharded.run_steps) that the multi-process tests drive
+    ev = [backend.event() for _ in range(steps + 1)]
     kinds = []
-    gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid).replace("GPU-", "")
-    sampler = ClockSampler(gpu_id) if rank == 0 else None
+
+    def on_launch(kind, t):
+        ev[len(kinds) + 1].record()
+        kinds.append(kind)
+
     if world > 1:
         dist.barrier()
-    torch.cuda.synchronize()
+    backend.synchronize()
     launches0 = ctx.qsr_launch_count()
+    wall0 = time.time()
     ev[0].record()
-    n_ev = 1
-    for t in range(steps):
-        if t + 1 in ends and not sharded_path:
-            ctx.qsr_local_step_sync(t, t + 1)     # last step of a round: step and averaging in one launch
-            ev[n_ev].record()
-            n_ev += 1
-            kinds.append("sync")
-            continue
-        if t + 1 in ends:
-            # sharded round end: last step fused with this rank's row sums, all-reduce, finish
-            ctx.qsr_local_step_partial(t, sums)
-            all_reduce(sums[:ctx.qsr_sync_sum_floats()])
-            ctx.qsr_sync_finish(sums, K_total, t + 1)
-            ev[n_ev].record()
-            n_ev += 1
-            kinds.append("sync")
-            continue
-        ctx.qsr_local_step(t)
-        ev[n_ev].record()
-        n_ev += 1
-        kinds.append("step")
-    torch.cuda.synchronize()
+    sharded.run_steps(ctx, 0, steps, ex, on_launch)
+    backend.synchronize()
+    wall1 = time.time()
     if world > 1:
         dist.barrier()
     launches = ctx.qsr_launch_count() - launches0
-    total_ms = ev[0].elapsed_time(ev[n_ev - 1])
-    clocks = sampler.stop() if sampler else None
-    gaps = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(n_ev - 1)])
+    assert len(kinds) == steps
+    total_ms = ev[0].elapsed_time(ev[steps])
+    clocks = sampler.stop(wall0, wall1) if sampler else None
+    gaps = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(steps)])
     kinds = np.array(kinds)
-    step_ms = float(gaps[kinds == "step"].mean())
+    step_ms = float(gaps[kinds == "step"].mean()) if (kinds == "step").any() else None
     n_syncs = int((kinds == "sync").sum())
     sync_ms = float(gaps[kinds == "sync"].mean()) if n_syncs else None
     # the stand-alone averaging kernel, outside the timed window (the window's rounds end in the fused launch)
@@ -334,109 +390,105 @@ def main():
     if world == 1:
         for _ in range(3):
             ctx.qsr_sync(steps)
-        sa0, sa1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sa0, sa1 = backend.event(), backend.event()
         sa0.record()
         for _ in range(20):
             ctx.qsr_sync(steps)
         sa1.record()
-        torch.cuda.synchronize()
+        backend.synchronize()
         sync_alone_ms = sa0.elapsed_time(sa1) / 20
     ctx.close()
 
-    if world > 1:
-        tmax = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        total_ms = float(tmax.item())
+    total_ms = max_over_ranks(total_ms, backend)
     value = K_total * w.P * steps / (total_ms * 1e-3)
 
     # ---- end to end from host memory
     e2e = None
     if not args.no_e2e:
-        theta0_h = torch.zeros(w.P, dtype=torch.float32).pin_memory()
-        lam_p = torch.from_numpy(lam_h).pin_memory()
-        ths_p = torch.from_numpy(ths_h).pin_memory()
-        out_h = torch.empty(w.P, dtype=torch.float32).pin_memory()
+        theta0_h = backend.pinned(n=w.P)
+        lam_p = backend.pinned(lam_h)
+        ths_p = backend.pinned(ths_h)
+        out_h = backend.pinned(n=w.P)
         t_end = min(w.T, steps)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0, e1 = backend.event(), backend.event()
         if not sharded_path:
             # the slabs above are released first: qsr_train_host works in one caller-owned workspace
             theta = s1 = s2 = None
-            torch.cuda.empty_cache()
-            ws = torch.empty(B.qsr_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
-            torch.cuda.synchronize()
+            backend.release_cached_memory()
+            ws = backend.empty_bytes(B.qsr_workspace_bytes(cfg))
+            backend.synchronize()
             e0.record()
-            r_st, r_H, _ = B.qsr_train_host(cfg, theta0_h, lam_p, ths_p, out_h, ws, t_end=t_end, stream=stream)
+            r_st, r_H, _ = backend.train_host(cfg, theta0_h, lam_p, ths_p, out_h, ws, t_end)
             e1.record()
-            torch.cuda.synchronize()
+            backend.synchronize()
             e2e_ms = e0.elapsed_time(e1)
             done = int(r_st[-1] + r_H[-1])      # whole rounds: stops at the first round end at or after t_end
         else:
             if world > 1:
                 dist.barrier()
-            torch.cuda.synchronize()
+            backend.synchronize()
             e0.record()
             lam[:w.P].copy_(lam_p, non_blocking=True)
             ths[:w.P].copy_(ths_p, non_blocking=True)
-            theta0_d = torch.empty(P4, device=dev)
+            theta0_d = backend.zeros(P4)
             theta0_d[:w.P].copy_(theta0_h, non_blocking=True)
             s1.zero_()
             if s2 is not None:
                 s2.zero_()
-            ctx = B.Context(cfg, theta, s1, s2, lam, ths, stream=stream)
+            ctx = backend.context(cfg, theta, s1, s2, lam, ths)
             ctx.qsr_set_params(theta0_d)
-            n_sum = ctx.qsr_sync_sum_floats()
-            rounds = sharded.run_rounds(ctx, sums, K_total, 0, t_end, lambda buf: all_reduce(buf[:n_sum]))
+            rounds = sharded.run_steps(ctx, 0, t_end, ex, whole_rounds=True)
             out_h.copy_(theta[0, :w.P], non_blocking=True)
             e1.record()
-            torch.cuda.synchronize()
+            backend.synchronize()
             ctx.close()
             done = rounds[-1][0] + rounds[-1][1]
-            e2e_ms = e0.elapsed_time(e1)
             if world > 1:
                 dist.barrier()
-                tmax = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-                dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-                e2e_ms = float(tmax.item())
+            e2e_ms = max_over_ranks(e0.elapsed_time(e1), backend)
         e2e = {"value": K_total * w.P * done / (e2e_ms * 1e-3), "unit": UNIT, "steps": done,
+               "note": "a whole number of rounds: the run stops at the first round end at or after --steps",
                "h2d_bytes_per_step": 3 * w.P * 4 / done, "d2h_bytes_per_step": w.P * 4 / done,
-               "api": "sharded.run_rounds" if sharded_path else "qsr_train_host"}
+               "api": "sharded.run_steps" if sharded_path else "qsr_train_host"}
 
     if rank != 0:
-        dist.destroy_process_group()
-        return
+        return None
 
     peak, peak_kind = measured_peak()
-    step_bytes = step_bytes_per_update(w) * K_local * w.P
-    step_gbs = step_bytes / (step_ms * 1e-3) / 1e9
-    traffic = None
     n_slabs = 3 if w.opt == W.OPT_ADAMW else 2
     streams_from_hbm = n_slabs * K_local * P4 * 4 > 2 * L2_BYTES     # else the slabs stay in L2 and DRAM sees little
-    if NCU_TRAFFIC["step_source_sha256"] == step_source_hash() and streams_from_hbm:
-        traffic = NCU_TRAFFIC["bytes_per_update"][w.opt] * K_local * w.P
-    roofline = {"bound": "hbm", "kernel": "local_step_kernel", "achieved": step_gbs, "peak": peak, "unit": "GB/s",
-                "frac": step_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
-                "frac_of_nominal_8TBps": step_gbs / NOMINAL_HBM_GBS,
-                "algorithmic_bytes_per_launch": step_bytes, "avg_launch_ms": step_ms}
-    kernels = {"local_step": {"launches": int((kinds == "step").sum()), "avg_ms": step_ms, "GBps": step_gbs,
-                              "frac_of_measured": step_gbs / peak}}
-    if sync_ms is not None and not sharded_path:
-        # fused: the round's last step also averages; its traffic is that of a plain step
-        fused_gbs = step_bytes / (sync_ms * 1e-3) / 1e9
-        kernels["local_step_with_mean"] = {"launches": n_syncs, "avg_ms": sync_ms, "GBps": fused_gbs,
-                                           "frac_of_measured": fused_gbs / peak,
-                                           "note": "last step of a round + replica averaging in one launch"}
+    kernels = {}
+    roofline = None
+    if step_ms is not None:
+        step_bytes = step_bytes_per_update(w) * K_local * w.P
+        step_gbs = step_bytes / (step_ms * 1e-3) / 1e9
+        traffic = None
+        if NCU_TRAFFIC["step_source_sha256"] == step_source_hash() and streams_from_hbm:
+            traffic = NCU_TRAFFIC["bytes_per_update"][w.opt] * K_local * w.P
+        roofline = {"bound": "hbm", "kernel": "local_step_kernel", "achieved": step_gbs, "peak": peak, "unit": "GB/s",
+                    "frac": step_gbs / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                    "frac_of_nominal_8TBps": step_gbs / NOMINAL_HBM_GBS,
+                    "algorithmic_bytes_per_launch": step_bytes, "avg_launch_ms": step_ms}
+        kernels["local_step"] = {"launches": int((kinds == "step").sum()), "avg_ms": step_ms, "GBps": step_gbs,
+                                 "frac_of_measured": step_gbs / peak}
+        if sync_ms is not None and not sharded_path:
+            # fused: the round's last step also averages; its traffic is that of a plain step
+            fused_gbs = step_bytes / (sync_ms * 1e-3) / 1e9
+            kernels["local_step_with_mean"] = {"launches": n_syncs, "avg_ms": sync_ms, "GBps": fused_gbs,
+                                               "frac_of_measured": fused_gbs / peak,
+                                               "note": "last step of a round + replica averaging in one launch"}
+        if sync_ms is not None and sharded_path:
+            # last step without the theta write-back, [P] sums out, then sums in and K rows written
+            end_bytes = step_bytes - 4.0 * K_local * w.P + 8.0 * w.P + 4.0 * K_local * w.P
+            end_gbs = end_bytes / (sync_ms * 1e-3) / 1e9
+            kernels["sharded_round_end"] = {"launches": n_syncs, "avg_ms": sync_ms, "GBps": end_gbs,
+                                            "frac_of_measured": end_gbs / peak,
+                                            "note": "last step fused with row sums + NCCL all-reduce of P floats + finish kernel"}
     if sync_alone_ms is not None:
         sa_gbs = 8.0 * K_local * w.P / (sync_alone_ms * 1e-3) / 1e9
         kernels["sync"] = {"launches_outside_window": 20, "avg_ms": sync_alone_ms, "GBps": sa_gbs,
                            "frac_of_measured": sa_gbs / peak, "frac_of_nominal_8TBps": sa_gbs / NOMINAL_HBM_GBS,
                            "note": "stand-alone replica-mean kernel (used when the state is averaged or reset)"}
-    if sync_ms is not None and sharded_path:
-        # last step without the theta write-back, [P] sums out, then sums in and K rows written
-        end_bytes = step_bytes - 4.0 * K_local * w.P + 8.0 * w.P + 4.0 * K_local * w.P
-        end_gbs = end_bytes / (sync_ms * 1e-3) / 1e9
-        kernels["sharded_round_end"] = {"launches": n_syncs, "avg_ms": sync_ms, "GBps": end_gbs,
-                                        "frac_of_measured": end_gbs / peak,
-                                        "note": "last step fused with row sums + NCCL all-reduce of P floats + finish kernel"}
 
     slab_bytes = n_slabs * K_local * P4 * 4
     l2_note = ("inputs larger than L2 (every launch streams the whole slabs)" if streams_from_hbm else
@@ -454,12 +506,28 @@ def main():
                    "parallelism": f"replica-sharded dp{world}" if sharded_path else "1 GPU, replicas as slab rows"},
         "roofline": roofline, "kernels": kernels, "gpu_launches": int(launches), "clocks": clocks,
     }
+    if clocks and clocks.get("sm_mhz"):
+        # time x clock: equal products at different clocks mean the difference is the clock's (the power cap's)
+        out["sm_mhz_x_ms_per_step"] = clocks["sm_mhz"] * total_ms / steps
     if e2e is not None:
         out["e2e"] = e2e
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(base)
-    print(json.dumps(out))
+    return out
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    backend = CudaBackend(int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), world)
+    out = run_ours(args, backend)
+    if out is not None:
+        print(json.dumps(out))
     if world > 1:
+        import torch.distributed as dist
         dist.destroy_process_group()
 
 

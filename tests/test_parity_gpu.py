@@ -271,6 +271,70 @@ def test_sharded_sync_equals_single_process():
             ctx.close()
 
 
+class _TwoShards:
+    """Two contexts on one GPU behind the interface of one engine: every call goes to both, each shard writes its
+    partial sums to its own half of the buffer, and the 'all-reduce' adds the halves, as the exchange would."""
+
+    def __init__(self, parts, n_sum):
+        self.parts, self.n = parts, n_sum
+
+    def qsr_round_length(self, t):
+        H = {ctx.qsr_round_length(t) for _, ctx in self.parts}
+        assert len(H) == 1
+        return H.pop()
+
+    def qsr_local_step(self, t):
+        for _, ctx in self.parts:
+            ctx.qsr_local_step(t)
+
+    def qsr_local_step_partial(self, t, sums):
+        for r, (_, ctx) in enumerate(self.parts):
+            ctx.qsr_local_step_partial(t, sums[r * self.n:(r + 1) * self.n])
+
+    def all_reduce(self, sums):
+        total = sums[:self.n] + sums[self.n:]
+        sums[:self.n] = total
+        sums[self.n:] = total
+
+    def qsr_sync_finish(self, sums, K_total, t_next):
+        for r, (_, ctx) in enumerate(self.parts):
+            ctx.qsr_sync_finish(sums[r * self.n:(r + 1) * self.n], K_total, t_next)
+
+
+@pytest.mark.parametrize("mode", [W.STATE_KEEP, W.STATE_AVERAGE, W.STATE_RESET])
+@pytest.mark.parametrize("opt", [W.OPT_SGDM, W.OPT_ADAMW])
+def test_sharded_loop_over_two_contexts(opt, mode):
+    """The product's round loop (sharded.run_steps, the one the benchmark times and the gloo tests drive) over the
+    library's own partial-sum and finish launches: 7 workers split 4 + 3 over two contexts, all state modes -- in
+    AVERAGE mode the exchanged buffer carries the sums of the state slabs after those of the parameters."""
+    from paper_2310_14423_b200 import sharded
+    w = W.tiny_workload(opt, K=7, P=2003, T=40, state_sync=mode)
+    lam, ths, lam_d, ths_d = G.device_inputs(w)
+    parts = []
+    for r in range(2):
+        rows, k0 = sharded.shard(7, 2, r)
+        S = G.Slabs(w, K=rows)
+        parts.append((S, G.make_context(w, S, lam_d, ths_d, worker_offset=k0)))
+    n_sum = parts[0][1].qsr_sync_sum_floats()
+    assert n_sum == (1 if mode != W.STATE_AVERAGE else (3 if opt == W.OPT_ADAMW else 2)) * 2004
+    pair = _TwoShards(parts, n_sum)
+    sums = torch.zeros(2 * n_sum, device="cuda")
+    rounds = sharded.run_steps(pair, 0, w.T, sharded.Exchange(sums, 7, pair.all_reduce), whole_rounds=True)
+    torch.cuda.synchronize()
+    orc = G.oracle_on(w, lam, ths)
+    ost, oH = orc.run()
+    assert [r[0] for r in rounds] == ost.tolist() and [r[1] for r in rounds] == oH.tolist()
+    for r, (S, ctx) in enumerate(parts):
+        rows, k0 = sharded.shard(7, 2, r)
+        assert G.rel_err(S.theta[:, :w.P].cpu().numpy(), orc.theta[k0:k0 + rows]) <= G.REL_TOL
+        if mode == W.STATE_AVERAGE:
+            assert G.rel_err(S.s1[:, :w.P].cpu().numpy(), orc.s1[k0:k0 + rows]) <= 1e-4
+        if mode == W.STATE_RESET:
+            assert not S.s1[:, :w.P].any()
+        assert S.guards_intact()
+        ctx.close()
+
+
 def test_train_host_equals_context_path():
     for opt in (W.OPT_SGDM, W.OPT_ADAMW):
         w = W.tiny_workload(opt, K=4, P=10007, T=50)

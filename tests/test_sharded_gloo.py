@@ -1,8 +1,10 @@
 """The replica-sharded round loop on CPU: two (and three) gloo ranks, each holding a block of workers.
 
-The loop under test is the product's (`sharded.run_rounds`, round lengths from the library's host schedule); the
-arithmetic of each rank is supplied by the CPU oracle standing in for the CUDA context, and the exchange is a real
-gloo all-reduce.  The result must equal a single-process oracle run over all K workers: same rounds, same
+The loop under test is the product's (`sharded.run_rounds`, i.e. `sharded.run_steps`, round lengths from the library's
+host schedule); the arithmetic of each rank is supplied by the CPU oracle standing in for the CUDA context, and the
+exchange is a real gloo all-reduce.  What this covers is the sequencing, the schedule and the layout of the exchanged
+buffer; the library's own partial-sum and finish kernels are covered on one GPU (test_parity_gpu.py drives the same
+loop over two real contexts).  The result must equal a single-process oracle run over all K workers: same rounds, same
 parameters (up to the summation order of the mean)."""
 import os
 import socket
@@ -21,12 +23,21 @@ from paper_2310_14423_b200 import workloads as W
 
 
 class OracleEngine:
-    """The methods `run_rounds` needs, over the oracle's rows k0 .. k0+rows-1."""
+    """The methods `run_rounds` needs, over the oracle's rows k0 .. k0+rows-1.  The partial sums use the library's
+    layout: the parameter sums first, then (state mode AVERAGE) those of state1 and state2, each region starting at a
+    multiple of P rounded up to 4 floats."""
 
     def __init__(self, w, lam, ths, rows, k0):
         self.w = w
         self.cfg = B.make_config(w, K=rows, worker_offset=k0)
         self.S = O.State(w, lam, ths, rows=rows, k0=k0)
+        self.P4 = (w.P + 3) // 4 * 4
+        self.arrays = [self.S.theta]
+        if w.state_sync == W.STATE_AVERAGE:
+            self.arrays += [self.S.s1] + ([self.S.s2] if w.opt == W.OPT_ADAMW else [])
+
+    def qsr_sync_sum_floats(self):
+        return len(self.arrays) * self.P4
 
     def qsr_round_length(self, t):
         return B.qsr_config_round_length(self.cfg, t)
@@ -36,10 +47,13 @@ class OracleEngine:
 
     def qsr_local_step_partial(self, t, sums):
         self.S.local_step(t)
-        sums.copy_(torch.from_numpy(self.S.theta.sum(axis=0)))
+        sums.zero_()
+        for a, x in enumerate(self.arrays):
+            sums[a * self.P4:a * self.P4 + self.w.P] = torch.from_numpy(x.sum(axis=0))
 
     def qsr_sync_finish(self, sums, K_total, t_next):
-        self.S.theta[:] = sums.numpy() / K_total
+        for a, x in enumerate(self.arrays):
+            x[:] = sums[a * self.P4:a * self.P4 + self.w.P].numpy() / K_total
         if self.w.state_sync == W.STATE_RESET:
             self.S.s1[:] = 0
             self.S.s2[:] = 0
@@ -60,9 +74,11 @@ def _rank_main(rank, world, port, opt, mode, K_total, out_dir):
         lam, ths = W.draw_inputs(w.P, w.data_seed)
         rows, k0 = sharded.shard(K_total, world, rank)
         eng = OracleEngine(w, lam, ths, rows, k0)
-        sums = torch.zeros(w.P, dtype=torch.float64)
+        sums = torch.zeros(eng.qsr_sync_sum_floats(), dtype=torch.float64)
         rounds = sharded.run_rounds(eng, sums, K_total, 0, w.T, lambda buf: dist.all_reduce(buf))
         np.save(os.path.join(out_dir, f"theta_{rank}.npy"), eng.S.theta)
+        np.save(os.path.join(out_dir, f"s1_{rank}.npy"), eng.S.s1)
+        np.save(os.path.join(out_dir, f"s2_{rank}.npy"), eng.S.s2)
         np.save(os.path.join(out_dir, f"rounds_{rank}.npy"), np.asarray(rounds, np.int64))
     finally:
         dist.destroy_process_group()
@@ -88,6 +104,9 @@ def test_shard_blocks_cover_all_workers():
     (2, 6, W.OPT_ADAMW, W.STATE_KEEP),
     (2, 4, W.OPT_SGDM, W.STATE_KEEP),
     (3, 7, W.OPT_ADAMW, W.STATE_RESET),
+    (2, 6, W.OPT_ADAMW, W.STATE_AVERAGE),        # three regions in the exchanged buffer
+    (3, 7, W.OPT_ADAMW, W.STATE_AVERAGE),        # uneven shards: 3 + 2 + 2 workers
+    (3, 7, W.OPT_SGDM, W.STATE_AVERAGE),         # two regions
 ])
 def test_sharded_rounds_equal_single_process(tmp_path, world, K_total, opt, mode):
     port = _free_port()
@@ -103,3 +122,5 @@ def test_sharded_rounds_equal_single_process(tmp_path, world, K_total, opt, mode
         rows, k0 = sharded.shard(K_total, world, r)
         assert theta.shape[0] == rows
         np.testing.assert_allclose(theta, ref.theta[k0:k0 + rows], rtol=1e-12, atol=1e-14)
+        np.testing.assert_allclose(np.load(tmp_path / f"s1_{r}.npy"), ref.s1[k0:k0 + rows], rtol=1e-12, atol=1e-14)
+        np.testing.assert_allclose(np.load(tmp_path / f"s2_{r}.npy"), ref.s2[k0:k0 + rows], rtol=1e-12, atol=1e-14)
