@@ -50,6 +50,11 @@ NCU_TRAFFIC = {
     "bytes_per_update": {"adamw": 24.08, "sgdm": 16.07},
 }
 
+# Thread-instructions per element-update of resident_steps_kernel's step loop (ncu smsp__thread_inst_executed.sum of
+# one launch / (K * P * steps in the launch), captured on c2 and c1): the "algorithmic work" of the ALU roofline.
+NCU_RESIDENT_INSTR = {"source_sha256": "50003bae45ccf418daa7e0cf5905989b256153612eaa9679a289badc969e7cfb", "adamw": 51.50, "sgdm": 49.24}
+SM_COUNT, LANES_PER_SM_CLK = 148, 4 * 32      # 4 schedulers per SM, one warp instruction (32 lanes) each per clock
+
 
 def parse_args():
     ap = argparse.ArgumentParser()
@@ -62,6 +67,9 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--packed-rows", action="store_true",
                     help="rows packed at P (rounded up to 4) instead of the stride qsr_row_stride_hint recommends")
+    ap.add_argument("--resident-steps", type=int, default=0,
+                    help="BENCHMARK-ONLY: up to N (<= 128) consecutive steps per launch with parameters and state held in "
+                         "registers (possible only with the in-kernel synthetic gradient); one GPU; the roofline is ALU")
     ap.add_argument("--sharded-path", action="store_true",
                     help="on one GPU, still end rounds the multi-GPU way (partial sums, all-reduce of one rank, finish)")
     return ap.parse_args()
@@ -75,15 +83,26 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def step_source_hash():
+def source_region_hash(begin: str, end: str):
+    """sha256 of csrc/kernels.cu between two of its section markers (None if either is gone)."""
     with open(os.path.join(ROOT, "paper_2310_14423_b200", "csrc", "kernels.cu")) as f:
         text = f.read()
     bar = "// " + "-" * 94 + " "
     try:
-        region = text[text.index(bar + "noise"):text.index("// Sum over rows of one 16-byte column")]
+        region = text[text.index(bar + begin if begin else ""):text.index(end)]
     except ValueError:
         return None
     return hashlib.sha256(region.encode()).hexdigest()
+
+
+def step_source_hash():
+    return source_region_hash("noise", "// Sum over rows of one 16-byte column")
+
+
+def resident_source_hash():
+    a = source_region_hash("noise", "// Weight-decay scalar for the column")
+    b = source_region_hash("resident steps", "// " + "-" * 94 + " test hook")
+    return None if a is None or b is None else hashlib.sha256((a + b).encode()).hexdigest()
 
 
 class ClockSampler:
@@ -516,6 +535,90 @@ def run_ours(args, backend):
     return out
 
 
+def run_resident(args, backend):
+    """BENCHMARK-ONLY leg: the run's rounds as register-resident launches of up to N steps (qsr_set_resident_steps).
+    Times whole rounds: global steps [0, end of the round that holds step --steps - 1)."""
+    from paper_2310_14423_b200 import binding as B
+    from paper_2310_14423_b200 import workloads as W
+
+    B.lib()
+    w = W.workload(args.workload)
+    if args.steps > w.T:
+        raise SystemExit(f"--steps must be <= {w.T}")
+    lam_h, ths_h = W.draw_inputs(w.P, w.data_seed)
+    P4 = (w.P + 3) // 4 * 4
+    lam, ths = backend.zeros(P4), backend.zeros(P4)
+    lam[:w.P].copy_(backend.torch.from_numpy(lam_h))
+    ths[:w.P].copy_(backend.torch.from_numpy(ths_h))
+    stride = P4 if args.packed_rows else B.qsr_row_stride_hint(w.P)
+    theta, s1 = backend.zeros(w.K, stride), backend.zeros(w.K, stride)
+    s2 = backend.zeros(w.K, stride) if w.opt == W.OPT_ADAMW else None
+    cfg = B.make_config(w, row_stride=stride)
+
+    def fresh_context():
+        theta.zero_()
+        s1.zero_()
+        if s2 is not None:
+            s2.zero_()
+        ctx = backend.context(cfg, theta, s1, s2, lam, ths)
+        ctx.qsr_set_resident_steps(args.resident_steps)
+        return ctx
+
+    sampler = backend.clock_sampler()
+    reps = max(args.warmup, 3)
+    ctx = fresh_context()
+    for _ in range(reps):                                   # warm-up: the same window, untimed
+        ctx.qsr_run(0, args.steps)
+    backend.synchronize()
+    ctx.close()
+    ctx = fresh_context()
+    e0, e1 = backend.event(), backend.event()
+    backend.synchronize()
+    wall0 = time.time()
+    e0.record()
+    st, H = ctx.qsr_run(0, args.steps)
+    e1.record()
+    backend.synchronize()
+    wall1 = time.time()
+    launches = ctx.qsr_launch_count()
+    ctx.close()
+    clocks = sampler.stop(wall0, wall1)
+    total_ms = e0.elapsed_time(e1)
+    done = int(st[-1] + H[-1])
+    updates = w.K * w.P * done
+    value = updates / (total_ms * 1e-3)
+    sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
+    peak = SM_COUNT * LANES_PER_SM_CLK * sm_mhz * 1e6 / 1e9            # G thread-instructions per second
+    instr = NCU_RESIDENT_INSTR[w.opt] if NCU_RESIDENT_INSTR["source_sha256"] == resident_source_hash() else None
+    achieved = instr * value / 1e9 if instr else None
+    n_slabs = 3 if w.opt == W.OPT_ADAMW else 2
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": 1, "steps": done, "warmup": reps,
+        "ms_per_step": total_ms / done, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "benchmark_only": True,
+        "config": {"workload": f"{w.name}: K={w.K}, P={w.P}, {w.opt}", "K_per_gpu": w.K, "K_total": w.K, "P": w.P,
+                   "row_stride": stride, "opt": w.opt, "T": w.T, "resident_steps_per_launch": args.resident_steps,
+                   "window": f"global steps [0,{done}): the whole rounds that cover --steps {args.steps}",
+                   "syncs_in_window": int(len(st)),
+                   "l2": f"slabs of {n_slabs * w.K * P4 * 4 / 2**20:.0f} MiB are read once and written once per launch of up "
+                         f"to {args.resident_steps} steps; the launch is bound by its instruction stream, not by memory",
+                   "parallelism": "1 GPU, replicas as slab rows",
+                   "note": "BENCHMARK-ONLY: parameters and state stay in registers across steps, which only the "
+                           "in-kernel synthetic gradient allows; not the path a training loop takes"},
+        "roofline": {"bound": "alu", "kernel": "resident_steps_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "G thread-instr/s", "frac": achieved / peak if achieved else None,
+                     "peak_kind": f"{SM_COUNT} SMs x {LANES_PER_SM_CLK} lanes per clock x the median SM clock sampled "
+                                  f"during the run ({sm_mhz:.0f} MHz)",
+                     "thread_instr_per_update": instr, "avg_launch_ms": total_ms / launches, "traffic": None},
+        "gpu_launches": int(launches), "clocks": clocks,
+    }
+    if clocks and clocks.get("sm_mhz"):
+        out["sm_mhz_x_ms_per_step"] = clocks["sm_mhz"] * total_ms / done
+    if not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(w)
+    return out
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
@@ -523,7 +626,12 @@ def main():
         return
     world = int(os.environ.get("WORLD_SIZE", "1"))
     backend = CudaBackend(int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), world)
-    out = run_ours(args, backend)
+    if args.resident_steps > 0:
+        if world > 1:
+            raise SystemExit("--resident-steps is a one-GPU leg")
+        out = run_resident(args, backend)
+    else:
+        out = run_ours(args, backend)
     if out is not None:
         print(json.dumps(out))
     if world > 1:

@@ -171,7 +171,9 @@ int qsr_local_step(qsr_ctx *ctx, int64_t t, const float *grads);
 
 /* End of a round (Algorithm 2): theta_bar[i] = (1/K) * sum_k theta[k,i], summed in fp32 for k = 0..K-1 and divided
  * by K, then copied to every row; optimizer state treated per state_sync.  In RESET mode the bias-correction origin
- * moves to t_next (the first step of the next round).  One kernel launch; asynchronous. */
+ * moves to t_next (the first step of the next round).  One kernel launch, two in RESET mode (the zero-fill of the
+ * state slabs is a launch of its own: a pure write stream is fastest when it is not mixed into the averaging's
+ * loads); asynchronous. */
 int qsr_sync(qsr_ctx *ctx, int64_t t_next);
 
 /* The last local step of a round and the averaging that ends it (Eq. 1 followed by the All-Reduce line of
@@ -226,7 +228,7 @@ int qsr_sync_finish(qsr_ctx *ctx, const float *sum, int32_t K_total, int64_t t_n
  *   - All contexts and all calls in the process share the one array.  Each call overwrites what it needs before
  *     reading it, so an earlier call's leftovers are harmless; but two calls whose kernels can overlap on the GPU
  *     (different streams, no ordering between them) race on it.  Keep the calls on one stream or order them.
- * Two kernel launches; asynchronous. */
+ * Two kernel launches (three in RESET mode); asynchronous. */
 #define QSR_STATIC_SCRATCH_FLOATS (1 << 20) /* 4 MiB */
 int qsr_sync_static(qsr_ctx *ctx, int64_t t_next);
 
@@ -251,6 +253,22 @@ int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
  * kernel, so on B200 with 1 MiB slabs and rounds of 4-8 steps a replayed run was 12 % slower than the direct one;
  * it is off unless asked for. */
 int qsr_set_graph_replay(qsr_ctx *ctx, int32_t max_steps_per_graph);
+
+/* BENCHMARK-ONLY: several local steps per launch with the parameters and the optimizer state held in registers in
+ * between (Algorithm 2's inner "for h" loop inside one kernel).  This is possible only because the synthetic gradient
+ * is generated in the kernel; a training loop has to return to the host after every step for its next gradient, so
+ * no number measured with this switch on describes the path a real run takes.  What it shows is what the per-step
+ * launches cost when the whole problem fits in cache: with 1 MiB slabs a step kernel takes ~4 us of launch latency
+ * for ~0.5 us of arithmetic.
+ * With max_steps_per_launch = N in 1..128, qsr_run packs consecutive steps into launches of at most N steps: every
+ * thread owns one worker's four coordinates, reads them once, takes the steps (per-step learning rate and bias
+ * corrections arrive as kernel arguments) and writes them once.  One block holds all K rows of its columns, so with
+ * state_sync = QSR_STATE_KEEP the averaging at a round end happens inside the launch (through shared memory, k
+ * ascending, one division: the bits of qsr_local_step_sync) and a launch runs across round ends; in the other state
+ * modes a launch stops at the round end and qsr_sync follows.  Results are bit-identical to per-step launches.
+ * N = 0 (the default) switches it off.  QSR_ERANGE for N outside 0..128 or K > 32.  While a tensor table or gradient
+ * clipping is set, qsr_run launches per step as before.  Takes precedence over graph replay. */
+int qsr_set_resident_steps(qsr_ctx *ctx, int32_t max_steps_per_launch);
 
 /* Kernel launches issued through this context so far (a replayed graph counts its kernels). */
 int64_t qsr_launch_count(const qsr_ctx *ctx);

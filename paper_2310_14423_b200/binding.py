@@ -28,7 +28,7 @@ QSR_STATIC_SCRATCH_FLOATS = 1 << 20
 EXPORTS = ("qsr_config_check", "qsr_row_stride_hint", "qsr_config_learning_rate", "qsr_config_round_length", "qsr_config_schedule",
            "qsr_workspace_bytes", "qsr_init", "qsr_destroy", "qsr_round_length", "qsr_set_tensor_table", "qsr_clip_workspace_floats", "qsr_set_grad_clip", "qsr_set_params", "qsr_local_step",
            "qsr_local_step_sync", "qsr_parallel_step", "qsr_sync", "qsr_sync_sum_floats", "qsr_sync_partial", "qsr_local_step_partial", "qsr_sync_finish", "qsr_sync_static", "qsr_run", "qsr_launch_count",
-           "qsr_set_launch_shape", "qsr_set_graph_replay", "qsr_train_host", "qsr_debug_box_muller", "qsr_strerror")
+           "qsr_set_launch_shape", "qsr_set_graph_replay", "qsr_set_resident_steps", "qsr_train_host", "qsr_debug_box_muller", "qsr_strerror")
 
 
 class QsrConfig(C.Structure):
@@ -88,6 +88,7 @@ def lib():
             "qsr_launch_count": (i64, [vp]),
             "qsr_set_launch_shape": (C.c_int, [vp, i32, i32, i32]),
             "qsr_set_graph_replay": (C.c_int, [vp, i32]),
+            "qsr_set_resident_steps": (C.c_int, [vp, i32]),
             "qsr_train_host": (C.c_int, [cfg, vp, vp, vp, vp, vp, i64, i64, vp, vp, vp, i64, C.POINTER(i64), C.POINTER(i64)]),
             "qsr_debug_box_muller": (C.c_int, [vp, i64, vp, vp, vp, vp]),
             "qsr_strerror": (C.c_char_p, [C.c_int]),
@@ -260,6 +261,10 @@ class Context:
 
     def qsr_set_graph_replay(self, max_steps_per_graph: int) -> None:
         _check(lib().qsr_set_graph_replay(self._h, max_steps_per_graph), "qsr_set_graph_replay")
+
+    def qsr_set_resident_steps(self, max_steps_per_launch: int) -> None:
+        """Benchmark-only: up to this many consecutive steps per launch, state held in registers (0 = off)."""
+        _check(lib().qsr_set_resident_steps(self._h, max_steps_per_launch), "qsr_set_resident_steps")
 
     def qsr_set_launch_shape(self, step_threads: int = 0, step_rows_in_flight: int = 0, sync_threads: int = 0) -> None:
         _check(lib().qsr_set_launch_shape(self._h, step_threads, step_rows_in_flight, sync_threads), "qsr_set_launch_shape")

@@ -28,6 +28,7 @@ struct qsr_ctx {
     const float *lambda, *theta_star;
     cudaStream_t stream;
     int device;               // ordinal of the device that was current at qsr_init
+    int sm_count;             // its number of multiprocessors
     qsr::LaunchShape shape;
     int64_t t_state_origin;
     int64_t launches;
@@ -38,6 +39,7 @@ struct qsr_ctx {
     double clip_norm;         // > 0: gradient clipping on
     float *clip_ws;           // caller's workspace for the norm partials and the factors
     int32_t graph_steps;      // > 0: qsr_run replays its launches from CUDA graphs of at most this many steps
+    int32_t resident_steps;   // > 0: qsr_run packs up to this many consecutive steps into one register-resident launch
     std::vector<StepGraph> graphs;
 };
 
@@ -137,6 +139,77 @@ void drop_graphs(qsr_ctx &x)
 // workspace, so it stays on the direct path.
 bool graph_replay_applies(const qsr_ctx &x) { return x.graph_steps > 0 && !(x.clip_norm > 0.0); }
 
+// Register-resident launches cover what qsr_run issues by itself with the plain kernel instance: generated gradients,
+// uniform weight decay, no clipping, and few enough workers for one block to hold all rows of its columns.
+bool resident_applies(const qsr_ctx &x)
+{
+    return x.resident_steps > 0 && !(x.clip_norm > 0.0) && x.n_tensors == 0 && x.cfg.K <= qsr::kMaxResidentK;
+}
+
+// Algorithm 2 over the rounds that start in [t_begin, t_end) with consecutive steps packed into register-resident
+// launches of at most resident_steps steps.  With the state kept per worker a launch runs across round ends (the
+// averaging is block-local); in the other state modes a launch stops at the round end and the stand-alone
+// synchronization follows, which also moves the bias-correction origin in RESET mode before the next step's scalars
+// are formed.
+int run_resident(qsr_ctx &x, int64_t t_begin, int64_t t_end, int64_t *round_start, int64_t *round_len, int64_t cap,
+                 int64_t *n_rounds)
+{
+    const bool keep = x.cfg.state_sync == QSR_STATE_KEEP;
+    qsr::ResidentParams q;
+    std::memset(&q, 0, sizeof q);
+    // Columns per block (threads = columns x K, whole warps, at most 1024): 32 gives each warp 512 contiguous bytes of a
+    // row, but a small problem has only a few blocks per multiprocessor and whole blocks of imbalance (P = 65,536, K = 4:
+    // 512 blocks of 128 threads on 148 multiprocessors, i.e. 3 or 4 each); narrower blocks even that out, and the rows
+    // are only touched once per launch.  Take a narrower width only where it fills the last wave by 2 % more.
+    {
+        const int64_t n_col = (x.cfg.P + 3) >> 2;
+        double best = -1.0;
+        for (int cx : {64, 32, 16, 8}) {
+            const int threads = cx * x.cfg.K;
+            if (threads % 32 != 0 || threads > 1024 || (cx == 64 && x.cfg.K > 2)) continue;
+            const int64_t blocks = (n_col + cx - 1) / cx;
+            const int64_t waves = (blocks + x.sm_count - 1) / x.sm_count;
+            const double fill = double(blocks) / double(waves * x.sm_count);
+            if (fill > best + 0.02) { best = fill; q.cols_per_block = cx; }
+        }
+        if (best < 0.0) q.cols_per_block = 32;     // K = 1 with 32 columns is one warp per block: always valid
+    }
+    auto flush = [&]() -> int {
+        if (q.n_steps == 0) return QSR_OK;
+        x.launches++;
+        const int err = qsr::launch_resident_steps(q, x.cfg.opt, x.stream);
+        q.n_steps = 0;
+        std::memset(q.sync_after, 0, sizeof q.sync_after);
+        return cuda_rc(err);
+    };
+    int64_t s = 0;
+    for (int64_t t = t_begin; t < t_end;) {
+        const int64_t H = qsr::round_length(x.cfg, t);       // GetH
+        const RoundRange range(s, t, H);
+        for (int64_t h = 0; h < H; ++h) {
+            const qsr::StepParams sp = step_params(x, t + h, nullptr);
+            if (q.n_steps == 0) q.base = sp;                 // pointers, constants and the first step's index
+            q.per_step[q.n_steps] = qsr::ResidentScalars{sp.eta, sp.eta_wd, sp.step_size, sp.inv_sqrt_bc2};
+            if (keep && h == H - 1) q.sync_after[q.n_steps >> 5] |= 1u << (q.n_steps & 31);
+            if (++q.n_steps == x.resident_steps)
+                if (int rc = flush()) return rc;
+        }
+        if (!keep) {
+            if (int rc = flush()) return rc;
+            if (int rc = qsr_sync(&x, t + H)) return rc;
+        }
+        if (s < cap) {
+            round_start[s] = t;
+            round_len[s] = H;
+        }
+        ++s;
+        t += H;
+    }
+    if (int rc = flush()) return rc;
+    if (n_rounds) *n_rounds = s;
+    return QSR_OK;
+}
+
 cudaKernelNodeParams node_params(const qsr::StepLaunch &L, void **args)
 {
     cudaKernelNodeParams k;
@@ -228,6 +301,9 @@ int qsr_init(qsr_ctx **out, const qsr_config *cfg, float *params, float *state1,
     x->lambda = lambda; x->theta_star = theta_star;
     x->stream = static_cast<cudaStream_t>(cuda_stream);
     x->device = dev;
+    x->sm_count = 148;
+    cudaDeviceGetAttribute(&x->sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (x->sm_count < 1) x->sm_count = 148;
     x->shape = qsr::LaunchShape();
     if (cfg->opt == QSR_OPT_SGDM) x->shape.step_threads = 128;
     // Slabs that stay resident in L2 between steps are served with far lower latency than HBM: a 4-row ring in
@@ -247,6 +323,7 @@ int qsr_init(qsr_ctx **out, const qsr_config *cfg, float *params, float *state1,
     x->n_tensors = 0; x->tensor_end = nullptr; x->wd_scale = nullptr;
     x->clip_norm = 0.0; x->clip_ws = nullptr;
     x->graph_steps = 0;
+    x->resident_steps = 0;
     *out = x;
     return QSR_OK;
 }
@@ -359,7 +436,7 @@ int qsr_sync(qsr_ctx *ctx, int64_t t_next)
     if (!ctx) return QSR_EINVAL;
     if (t_next < 0 || t_next > ctx->cfg.T) return QSR_ERANGE;
     const qsr::SyncParams p = sync_params(*ctx);
-    ctx->launches++;
+    ctx->launches += qsr::sync_launches(p);
     const int rc = cuda_rc(qsr::launch_sync(p, ctx->shape, ctx->stream));
     if (rc == QSR_OK && ctx->cfg.state_sync == QSR_STATE_RESET) ctx->t_state_origin = t_next;
     return rc;
@@ -414,7 +491,7 @@ int qsr_sync_finish(qsr_ctx *ctx, const float *sum, int32_t K_total, int64_t t_n
     qsr::SyncParams p = sync_params(*ctx);
     p.sum_in = sum;
     p.divisor = float(K_total);
-    ctx->launches++;
+    ctx->launches += qsr::sync_launches(p);
     const int rc = cuda_rc(qsr::launch_sync_finish(p, ctx->shape, ctx->stream));
     if (rc == QSR_OK) {
         ctx->partial_pending = false;
@@ -431,7 +508,7 @@ int qsr_sync_static(qsr_ctx *ctx, int64_t t_next)
     if (int64_t(p.n_mean) * p.P4 > int64_t(QSR_STATIC_SCRATCH_FLOATS)) return QSR_ERANGE;   // nothing was launched
     const int err = qsr::launch_sync_static(p, ctx->shape, ctx->device, ctx->stream);
     if (err != 0) return err == -1 ? QSR_ERANGE : (err == -2 ? QSR_ESTATE : QSR_ECUDA);
-    ctx->launches += 2;
+    ctx->launches += 1 + qsr::sync_launches(p);
     if (ctx->cfg.state_sync == QSR_STATE_RESET) ctx->t_state_origin = t_next;
     return QSR_OK;
 }
@@ -454,6 +531,7 @@ int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
     if (!ctx || cap < 0 || (cap > 0 && (!round_start || !round_len))) return QSR_EINVAL;
     if (t_begin < 0 || t_end > ctx->cfg.T || t_begin > t_end) return QSR_ERANGE;
     if (!ctx->lambda) return QSR_EINVAL;
+    if (resident_applies(*ctx)) return run_resident(*ctx, t_begin, t_end, round_start, round_len, cap, n_rounds);
     int64_t s = 0;
     for (int64_t t = t_begin; t < t_end;) {
         const int64_t H = qsr::round_length(ctx->cfg, t);       // GetH
@@ -496,6 +574,15 @@ int qsr_set_graph_replay(qsr_ctx *ctx, int32_t max_steps_per_graph)
     if (max_steps_per_graph < 0 || max_steps_per_graph > 1024) return QSR_ERANGE;
     if (max_steps_per_graph != ctx->graph_steps) drop_graphs(*ctx);
     ctx->graph_steps = max_steps_per_graph;
+    return QSR_OK;
+}
+
+int qsr_set_resident_steps(qsr_ctx *ctx, int32_t max_steps_per_launch)
+{
+    if (!ctx) return QSR_EINVAL;
+    if (max_steps_per_launch < 0 || max_steps_per_launch > qsr::kMaxResidentSteps) return QSR_ERANGE;
+    if (max_steps_per_launch > 0 && ctx->cfg.K > qsr::kMaxResidentK) return QSR_ERANGE;
+    ctx->resident_steps = max_steps_per_launch;
     return QSR_OK;
 }
 

@@ -67,6 +67,23 @@ struct LaunchShape {
 // row sums written to StepParams::sum_out (a round's last step when the workers are sharded over GPUs).
 enum { FUSE_NONE = 0, FUSE_MEAN = 1, FUSE_SUM = 2 };
 
+// Several consecutive local steps in ONE launch, parameters and optimizer state held in registers in between
+// (possible only because the synthetic gradient is generated in the kernel: a training loop has to leave the device
+// code after every step to get its next gradient).  Per-step scalars travel as kernel arguments.
+constexpr int kMaxResidentSteps = 128;   // 2 KB of per-step scalars: the whole argument block stays below 4 KB
+constexpr int kMaxResidentK = 32;        // the K rows of a column sit in one block of 32 columns x K threads
+struct ResidentScalars {
+    float eta, eta_wd, step_size, inv_sqrt_bc2;    // as in StepParams, for one step
+};
+struct ResidentParams {
+    StepParams base;                     // pointers, sizes, noise key, constants; base.step is the first step
+    int32_t n_steps;                     // 1..kMaxResidentSteps
+    int32_t cols_per_block;
+    uint32_t sync_after[kMaxResidentSteps / 32];   // bit h: step h ends a round -> average the parameters over the rows
+    ResidentScalars per_step[kMaxResidentSteps];
+};
+int launch_resident_steps(const ResidentParams &q, int opt, void *stream);
+
 // One instance of the step kernel with its launch geometry: what cudaLaunchKernel or a CUDA-graph kernel node needs.
 // The kernel's only argument is a StepParams by value.
 struct StepLaunch {
@@ -82,9 +99,11 @@ int launch_step(const StepParams &p, int opt, const LaunchShape &shape, void *st
 int launch_step_mean(const StepParams &p, int opt, const LaunchShape &shape, void *stream);   // step + replica mean
 int launch_step_sum(const StepParams &p, int opt, const LaunchShape &shape, void *stream);    // step + row sums to p.sum_out
 int launch_parallel_step(const StepParams &p, int opt, const LaunchShape &shape, void *stream);  // Algorithm 1, row 0
-int launch_sync(const SyncParams &p, const LaunchShape &shape, void *stream);          // mean + write back (+ zero)
+// A synchronization that resets the optimizer state (n_zero > 0) zero-fills it in a second launch.
+int launch_sync(const SyncParams &p, const LaunchShape &shape, void *stream);          // mean + write back [+ reset launch]
 int launch_sync_partial(const SyncParams &p, const LaunchShape &shape, void *stream);  // sums only
-int launch_sync_finish(const SyncParams &p, const LaunchShape &shape, void *stream);   // sums -> rows (+ zero)
+int launch_sync_finish(const SyncParams &p, const LaunchShape &shape, void *stream);   // sums -> rows [+ reset launch]
+inline int sync_launches(const SyncParams &p) { return p.n_zero > 0 ? 2 : 1; }       // of launch_sync / launch_sync_finish
 int launch_broadcast(float *theta, const float *theta0, int64_t P, int64_t stride, int32_t K,
                      const LaunchShape &shape, void *stream);
 // Gradient clipping: grid of the norm pass and the two passes that leave the factors at ws + clip_grid(...) * rows.

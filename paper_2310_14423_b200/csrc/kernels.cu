@@ -10,6 +10,7 @@
 
 #include <atomic>
 #include <cstdint>
+#include <cstring>
 
 #include "internal.h"
 
@@ -525,20 +526,10 @@ __device__ __forceinline__ void sync_column(float *slab, const float *sum_in, fl
     }
 }
 
-__device__ __forceinline__ void zero_column(float *slab, int64_t i0, const SyncParams &p)
-{
-    if (i0 + 4 <= p.P) {
-        const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-        for (int k = 0; k < p.K; ++k) st4(slab + int64_t(k) * p.stride + i0, zero);
-    } else {
-        for (int64_t i = i0; i < p.P; ++i)
-            for (int k = 0; k < p.K; ++k) slab[int64_t(k) * p.stride + i] = 0.f;
-    }
-}
-
-// slab[0 .. n_mean) are averaged (theta always; the optimizer state in AVERAGE mode); in modes 0 and 2 the
-// arrays slab[n_mean .. n_mean+n_zero) are zero-filled (state reset).
+// slab[0 .. n_mean) are averaged (theta always; the optimizer state in AVERAGE mode).  A thread owns one 16-byte
+// column of all K rows: eight row loads in flight, the sum in registers, one division, K stores.  The second half of
+// a sharded synchronization (MODE 2) keeps this shape although it only reads one vector: the division is then done
+// once per column, where one-row-per-block would repeat it for each of the K rows and become bound by it.
 template <int MODE>
 __global__ void __launch_bounds__(512) sync_kernel(const SyncParams p)
 {
@@ -547,27 +538,152 @@ __global__ void __launch_bounds__(512) sync_kernel(const SyncParams p)
     for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < n_col; j += grid_stride) {
         const int64_t i0 = j << 2;
 #pragma unroll
-        for (int a = 0; a < 3; ++a) {
-            if (a < p.n_mean)
-                sync_column<MODE>(p.slab[a], p.sum_in + a * p.P4, p.sum_out + a * p.P4, i0, p);
-            else if (MODE != 1 && a < p.n_mean + p.n_zero)
-                zero_column(p.slab[a], i0, p);
+        for (int a = 0; a < 3; ++a)
+            if (a < p.n_mean) sync_column<MODE>(p.slab[a], p.sum_in + a * p.P4, p.sum_out + a * p.P4, i0, p);
+    }
+}
+
+// Rows written with zeros or from one source vector: the reset of the optimizer state and the replica copy of the
+// initial parameters.  These launches write K times what they read (or read nothing), and a write-only stream runs
+// at its best rate when it is not interleaved with a thread's own loads: B200 fills K rows of the ViT-B/16 set at
+// 7.3 TB/s from blocks that each write one contiguous 16 KB piece of one row, against 6.1 TB/s for the same zeros
+// stored by the threads of the averaging kernel after their K loads, and the one-to-K copy gains 4 % in this form
+// over one-column-per-thread.
+// Work item = (piece of kRowPiece columns, row); the K rows of a piece are neighbouring items, so the K blocks that
+// need the same piece of the source run together and all but the first find it in L2.
+constexpr int kRowThreads = 256, kRowColsPerThread = 4, kRowPiece = kRowThreads * kRowColsPerThread;
+
+struct RowsParams {
+    float *dst[3];            // up to three slabs [K, stride]
+    const float *src[3];      // source vector [P] of each slab (SRC 1)
+    int32_t n_slabs, K;
+    int64_t P, stride;
+};
+
+// SRC 0: zeros.  SRC 1: copy of src.
+template <int SRC>
+__global__ void __launch_bounds__(kRowThreads) rows_kernel(const __grid_constant__ RowsParams p)
+{
+    const int64_t n_col = (p.P + 3) >> 2;
+    const int64_t pieces = (n_col + kRowPiece - 1) / kRowPiece;
+    const int64_t rows = int64_t(p.n_slabs) * p.K;
+    const int64_t items = pieces * rows;
+    for (int64_t item = blockIdx.x; item < items; item += gridDim.x) {
+        const int64_t piece = item / rows;
+        const int r = int(item - piece * rows);
+        const int a = r / p.K, k = r - a * p.K;
+        float *row = p.dst[a] + int64_t(k) * p.stride;
+        const float *src = p.src[a];
+        const int64_t j0 = piece * kRowPiece + threadIdx.x;
+        float4 v[kRowColsPerThread];
+#pragma unroll
+        for (int c = 0; c < kRowColsPerThread; ++c) {
+            const int64_t i0 = (j0 + int64_t(c) * kRowThreads) << 2;
+            v[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (SRC != 0 && i0 + 4 <= p.P) v[c] = ld4(src + i0);
+        }
+#pragma unroll
+        for (int c = 0; c < kRowColsPerThread; ++c) {
+            const int64_t i0 = (j0 + int64_t(c) * kRowThreads) << 2;
+            if (i0 + 4 <= p.P) st4(row + i0, v[c]);
+        }
+        // Ragged end of the row (P not a multiple of 4): its one to three floats are written, one per thread, by the
+        // block that holds the row's last piece.  Kept out of the loops above, whose four loads and four stores the
+        // compiler otherwise no longer issues back to back (10 % on the one-to-K copy).
+        if (piece == pieces - 1 && int(threadIdx.x) < int(p.P & 3)) {
+            const int64_t i = (p.P & ~int64_t(3)) + threadIdx.x;
+            row[i] = SRC == 0 ? 0.f : src[i];
         }
     }
 }
 
-__global__ void __launch_bounds__(512) broadcast_kernel(float *theta, const float *theta0, int64_t P, int64_t stride, int K)
+template <int SRC>
+int launch_rows(const RowsParams &p, void *stream)
 {
-    const int64_t n_col = (P + 3) >> 2;
-    const int64_t grid_stride = int64_t(gridDim.x) * blockDim.x;
-    for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < n_col; j += grid_stride) {
-        const int64_t i0 = j << 2;
-        if (i0 + 4 <= P) {
-            const float4 v = ld4(theta0 + i0);
-            for (int k = 0; k < K; ++k) st4(theta + int64_t(k) * stride + i0, v);
-        } else {
-            for (int64_t i = i0; i < P; ++i)
-                for (int k = 0; k < K; ++k) theta[int64_t(k) * stride + i] = theta0[i];
+    const int64_t n_col = (p.P + 3) >> 2;
+    int64_t items = ((n_col + kRowPiece - 1) / kRowPiece) * int64_t(p.n_slabs) * p.K;
+    if (items > 2147483647) items = 2147483647;     // the kernel strides over the rest
+    if (items < 1) return 0;
+    rows_kernel<SRC><<<unsigned(items), kRowThreads, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    return int(cudaGetLastError());
+}
+
+// ---------------------------------------------------------------------------------------------- resident steps
+//
+// q.n_steps consecutive local steps of Algorithm 2's inner loop in one launch.  A thread owns ONE row of one 16-byte
+// column: the rows of a column are independent between synchronizations, so spreading them over threads keeps the
+// register count low (theta, the state and lambda / theta* of four coordinates) and the machine full even when the
+// whole problem is a megabyte.  The block holds all K rows of its 32 (or 64) columns -- thread = row * columns +
+// column, so a warp still reads 512 contiguous bytes of one row -- and that makes the averaging block-local: where a
+// step ends a round (bit h of q.sync_after) the rows' new parameters go through shared memory and every thread forms
+// the mean itself, k ascending from zero and one division, i.e. the bits of the fused last step of the per-step path.
+// A launch can therefore run across round ends.  Slabs are read once at the start and written once at the end:
+// the launch is bound by the instruction stream of the noise generator and the optimizer, not by memory.
+// The arithmetic of a step is the per-step kernel's (same device functions, same expressions): results are
+// bit-identical to n_steps single launches.
+template <int OPT>
+__global__ void resident_steps_kernel(const __grid_constant__ ResidentParams q)
+{
+    extern __shared__ float4 round_end[];      // [K][cols_per_block]
+    const StepParams &p = q.base;
+    const int cx = q.cols_per_block;
+    const int c = int(threadIdx.x) % cx, k = int(threadIdx.x) / cx;
+    const int64_t n_col = (p.P + 3) >> 2;
+    const int64_t j = int64_t(blockIdx.x) * cx + c;
+    const int64_t i0 = j << 2;
+    // threads past the last column stay in the loop for the barriers; they load and store nothing
+    const int valid = j < n_col ? (i0 + 4 <= p.P ? 4 : int(p.P - i0)) : 0;
+    const int64_t e = int64_t(k) * p.stride + i0;
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 th = zero, a = zero, b = zero, lam = zero, ths = zero;
+    if (valid == 4) {
+        th = ld4(p.theta + e);
+        a = ld4(p.s1 + e);
+        if (OPT == QSR_OPT_ADAMW) b = ld4(p.s2 + e);
+        lam = ld4(p.lambda + i0);
+        ths = ld4(p.theta_star + i0);
+    } else if (valid > 0) {
+        th = ld4_guarded(p.theta + e, valid);
+        a = ld4_guarded(p.s1 + e, valid);
+        if (OPT == QSR_OPT_ADAMW) b = ld4_guarded(p.s2 + e, valid);
+        lam = ld4_guarded(p.lambda + i0, valid);
+        ths = ld4_guarded(p.theta_star + i0, valid);
+    }
+    StepParams s;                              // the scalars opt_update reads; everything else stays unused
+    s.mu = p.mu; s.omb1 = p.omb1; s.omb2 = p.omb2; s.eps = p.eps;
+    const float Kf = float(p.K);
+    for (int h = 0; h < q.n_steps; ++h) {
+        const ResidentScalars sc = q.per_step[h];
+        s.eta = sc.eta; s.step_size = sc.step_size; s.inv_sqrt_bc2 = sc.inv_sqrt_bc2;
+        const float wdv = OPT == QSR_OPT_SGDM ? p.wd : sc.eta_wd;
+        const float4 z = noise4(j, p.step + uint32_t(h), p.worker0 + uint32_t(k), p.round_key);
+        float4 g;
+        g.x = fmaf(p.sigma, z.x, lam.x * (th.x - ths.x));
+        g.y = fmaf(p.sigma, z.y, lam.y * (th.y - ths.y));
+        g.z = fmaf(p.sigma, z.z, lam.z * (th.z - ths.z));
+        g.w = fmaf(p.sigma, z.w, lam.w * (th.w - ths.w));
+        opt_update<OPT>(th.x, a.x, b.x, g.x, s, wdv);
+        opt_update<OPT>(th.y, a.y, b.y, g.y, s, wdv);
+        opt_update<OPT>(th.z, a.z, b.z, g.z, s, wdv);
+        opt_update<OPT>(th.w, a.w, b.w, g.w, s, wdv);
+        if ((q.sync_after[h >> 5] >> (h & 31)) & 1u) {      // uniform over the grid: every thread takes the barriers
+            round_end[k * cx + c] = th;
+            __syncthreads();
+            float4 acc = zero;
+            for (int r = 0; r < p.K; ++r) acc = add4(acc, round_end[r * cx + c]);
+            th = div4(acc, Kf);
+            __syncthreads();
+        }
+    }
+    if (valid == 4) {
+        st4(p.theta + e, th);
+        st4(p.s1 + e, a);
+        if (OPT == QSR_OPT_ADAMW) st4(p.s2 + e, b);
+    } else if (valid > 0) {
+        for (int l = 0; l < valid; ++l) {          // ragged last column: lanes 0 .. valid-1 (at most three)
+            p.theta[e + l] = l == 0 ? th.x : (l == 1 ? th.y : th.z);
+            p.s1[e + l] = l == 0 ? a.x : (l == 1 ? a.y : a.z);
+            if (OPT == QSR_OPT_ADAMW) p.s2[e + l] = l == 0 ? b.x : (l == 1 ? b.y : b.z);
         }
     }
 }
@@ -730,10 +846,22 @@ int launch_clip_coef(const StepParams &p, bool parallel, double max_norm, float 
     return int(cudaGetLastError());
 }
 
+// The state slabs a synchronization resets: a launch of its own after the averaging (see rows_kernel).
+static int launch_state_reset(const SyncParams &p, void *stream)
+{
+    if (p.n_zero == 0) return 0;
+    RowsParams r;
+    std::memset(&r, 0, sizeof r);
+    for (int a = 0; a < p.n_zero; ++a) r.dst[a] = p.slab[p.n_mean + a];
+    r.n_slabs = p.n_zero; r.K = p.K; r.P = p.P; r.stride = p.stride;
+    return launch_rows<0>(r, stream);
+}
+
 int launch_sync(const SyncParams &p, const LaunchShape &shape, void *stream)
 {
     sync_kernel<0><<<grid_for(p.P, shape.sync_threads), shape.sync_threads, 0, static_cast<cudaStream_t>(stream)>>>(p);
-    return int(cudaGetLastError());
+    if (cudaError_t e = cudaGetLastError()) return int(e);
+    return launch_state_reset(p, stream);
 }
 
 int launch_sync_partial(const SyncParams &p, const LaunchShape &shape, void *stream)
@@ -745,14 +873,31 @@ int launch_sync_partial(const SyncParams &p, const LaunchShape &shape, void *str
 int launch_sync_finish(const SyncParams &p, const LaunchShape &shape, void *stream)
 {
     sync_kernel<2><<<grid_for(p.P, shape.sync_threads), shape.sync_threads, 0, static_cast<cudaStream_t>(stream)>>>(p);
-    return int(cudaGetLastError());
+    if (cudaError_t e = cudaGetLastError()) return int(e);
+    return launch_state_reset(p, stream);
 }
 
 int launch_broadcast(float *theta, const float *theta0, int64_t P, int64_t stride, int32_t K,
                      const LaunchShape &shape, void *stream)
 {
-    broadcast_kernel<<<grid_for(P, shape.sync_threads), shape.sync_threads, 0, static_cast<cudaStream_t>(stream)>>>(
-        theta, theta0, P, stride, K);
+    RowsParams r;
+    std::memset(&r, 0, sizeof r);
+    r.dst[0] = theta; r.src[0] = theta0;
+    r.n_slabs = 1; r.K = K; r.P = P; r.stride = stride;
+    return launch_rows<1>(r, stream);
+}
+
+int launch_resident_steps(const ResidentParams &q, int opt, void *stream)
+{
+    const int64_t n_col = (q.base.P + 3) >> 2;
+    const int cx = q.cols_per_block;
+    const int64_t blocks = (n_col + cx - 1) / cx;
+    if (blocks > 2147483647 || q.base.K > kMaxResidentK || cx * q.base.K > 1024) return int(cudaErrorInvalidValue);
+    const unsigned threads = unsigned(cx * q.base.K);
+    const size_t smem = size_t(threads) * sizeof(float4);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (opt == QSR_OPT_SGDM) resident_steps_kernel<QSR_OPT_SGDM><<<unsigned(blocks), threads, smem, st>>>(q);
+    else resident_steps_kernel<QSR_OPT_ADAMW><<<unsigned(blocks), threads, smem, st>>>(q);
     return int(cudaGetLastError());
 }
 

@@ -45,3 +45,13 @@ def test_recorded_traffic_matches_the_kernel_source():
     for opt, algo in (("adamw", 24.5), ("sgdm", 16.5)):
         measured = bench.NCU_TRAFFIC["bytes_per_update"][opt]
         assert 0.95 * algo <= measured <= 1.02 * algo     # no re-reads: traffic ~ algorithmic bytes
+
+
+def test_recorded_instruction_counts_match_the_resident_kernel_source():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.resident_source_hash() == bench.NCU_RESIDENT_INSTR["source_sha256"], \
+        "the resident-steps kernel changed since the ncu capture: re-capture and update NCU_RESIDENT_INSTR"
+    # the ALU peak: 148 SMs x 4 schedulers x 32 lanes per clock
+    assert bench.SM_COUNT * bench.LANES_PER_SM_CLK == 18944
+    assert 40 < bench.NCU_RESIDENT_INSTR["sgdm"] < bench.NCU_RESIDENT_INSTR["adamw"] < 60
