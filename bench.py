@@ -46,8 +46,8 @@ L2_BYTES = 126e6
 # once, so traffic grows in proportion to K*P).  Valid only for the kernel source it was taken from: the hash covers
 # the noise generator, the optimizer update and local_step_kernel in csrc/kernels.cu.
 NCU_TRAFFIC = {
-    "step_source_sha256": "6c2fa12f453d27aa841b9366d84720bff8d1390a3c74bc8ff30a60d58949601e",
-    "bytes_per_update": {"adamw": 24.08, "sgdm": 16.07},
+    "step_source_sha256": "13c8e9bbf1a3e1513a8fe05499fb1a8af37d6dd6d63d0dd8179b671fd4e665fe",
+    "bytes_per_update": {"adamw": 24.07, "sgdm": 16.07},
 }
 
 # Thread-instructions per element-update of resident_steps_kernel's step loop (ncu smsp__thread_inst_executed.sum of

@@ -79,6 +79,7 @@ qsr::StepParams step_params(const qsr_ctx &x, int64_t t, const float *grads)
     p.step_size = float(eta / bc1);
     p.inv_sqrt_bc2 = float(1.0 / std::sqrt(bc2));
     p.eps = float(c.eps);
+    p.inv_K = 1.0f / float(c.K);
     p.n_tensors = x.n_tensors; p.tensor_end = x.tensor_end; p.wd_scale = x.wd_scale;
     return p;
 }

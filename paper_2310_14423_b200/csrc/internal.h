@@ -32,6 +32,7 @@ struct StepParams {
     float step_size;          // AdamW: eta / (1 - beta1^n)
     float inv_sqrt_bc2;       // AdamW: 1 / sqrt(1 - beta2^n)
     float eps;
+    float inv_K;              // 1 / K (exact when K is a power of two)
     int32_t n_tensors;             // 0: uniform weight decay
     const int64_t *tensor_end;     // device [n_tensors]: one past each tensor's last coordinate, ascending
     const float *wd_scale;         // device [n_tensors]: factor on the weight decay of each tensor

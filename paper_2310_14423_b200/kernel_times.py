@@ -111,7 +111,8 @@ def main(argv=None):
     ctx.close()
     for mode, per in ((W.STATE_AVERAGE, 8 + 8 * (n_slabs - 1)), (W.STATE_RESET, 8 + 4 * (n_slabs - 1))):
         c = context(mode)
-        add(f"replica mean, state {mode}", timed(lambda: c.qsr_sync(t[0])), per * KP)
+        label = f"replica mean, state {mode}" + (" (mean launch + state-reset launch)" if mode == W.STATE_RESET else "")
+        add(label, timed(lambda: c.qsr_sync(t[0])), per * KP)
         c.close()
     theta0 = torch.zeros(stride, device=dev)[:w.P]
     c = context()
