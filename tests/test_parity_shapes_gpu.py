@@ -89,3 +89,58 @@ def test_k32_slab_beyond_32bit_indexing():
     assert st.tolist() == [0, 478] and H.tolist() == [478, 481]
     _compare(w, lam, ths, theta, st, H, t_end=500)
     assert bool((theta[31, :w.P] == theta[0, :w.P]).all())
+
+
+def test_k32_reset_and_replica_copy_at_full_size():
+    """K=32 at the paper's peak learning rate with the optimizer state reset at every synchronization, from a non-zero
+    theta_bar(0): the replica copy and the state-reset launches write rows whose element offsets need 64 bits; three
+    rounds of four steps, compared on the coordinate subset, and the state slabs must be zero everywhere afterwards."""
+    w = W.workload("c5").replace(eta_max=8e-3, state_sync=W.STATE_RESET)
+    lam, ths, lam_d, ths_d = G.device_inputs(w)
+    stride = B.qsr_row_stride_hint(w.P)
+    theta = torch.full((w.K, stride), 7.0, device="cuda")          # 7.0 marks what must be overwritten or left alone
+    s1 = torch.full((w.K, stride), 7.0, device="cuda")
+    s2 = torch.full((w.K, stride), 7.0, device="cuda")
+    s1[:, :w.P] = 0.0
+    s2[:, :w.P] = 0.0
+    gen = torch.Generator(device="cuda").manual_seed(3)
+    theta0 = torch.randn(w.P, device="cuda", generator=gen) * 0.1
+    ctx = B.Context(B.make_config(w, row_stride=stride), theta, s1, s2, lam_d, ths_d,
+                    stream=torch.cuda.current_stream().cuda_stream)
+    ctx.qsr_set_params(theta0)
+    torch.cuda.synchronize()
+    assert bool((theta[31, :w.P] == theta0).all()) and bool((theta[0, :w.P] == theta0).all())
+    st, H = ctx.qsr_run(0, 12)
+    torch.cuda.synchronize()
+    ctx.close()
+    assert st.tolist() == [0, 4, 8] and H.tolist() == [4, 4, 4]
+    idx = W.coordinate_subset(w.layout, N_SUBSET, seed=7)
+    orc = G.oracle_on(w, lam, ths, idx)
+    orc.theta[:] = theta0[torch.from_numpy(idx).cuda()].double().cpu().numpy()
+    orc.run(0, 12)
+    cols = theta[:, torch.from_numpy(idx).cuda()].cpu().numpy()
+    assert (cols == cols[0]).all()
+    assert G.rel_err(cols[0], orc.theta[0]) <= G.REL_TOL
+    assert not bool(s1[:, :w.P].any()) and not bool(s2[:, :w.P].any())          # reset: zero on every row
+    if stride > w.P:                                                            # padding is never written
+        assert bool((theta[:, w.P:] == 7.0).all()) and bool((s1[:, w.P:] == 7.0).all()) and bool((s2[:, w.P:] == 7.0).all())
+
+
+def test_k32_resident_launches_at_full_size():
+    """The register-resident launches (benchmark-only) on the K=32 slabs: 64-bit offsets, 1024-thread blocks (32 columns
+    x 32 rows); the first round of 478 steps in four launches, against the oracle on the coordinate subset."""
+    w = W.workload("c5")
+    lam, ths, lam_d, ths_d = G.device_inputs(w)
+    stride = B.qsr_row_stride_hint(w.P)
+    theta = torch.zeros(w.K, stride, device="cuda")
+    s1 = torch.zeros(w.K, stride, device="cuda")
+    s2 = torch.zeros(w.K, stride, device="cuda")
+    ctx = B.Context(B.make_config(w, row_stride=stride), theta, s1, s2, lam_d, ths_d,
+                    stream=torch.cuda.current_stream().cuda_stream)
+    ctx.qsr_set_resident_steps(128)
+    st, H = ctx.qsr_run(0, 400)
+    torch.cuda.synchronize()
+    assert ctx.qsr_launch_count() == 4 and st.tolist() == [0] and H.tolist() == [478]
+    ctx.close()
+    _compare(w, lam, ths, theta, st, H, t_end=400)
+    assert bool((theta[31, :w.P] == theta[0, :w.P]).all())
