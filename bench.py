@@ -51,8 +51,11 @@ NCU_TRAFFIC = {
 }
 
 # Thread-instructions per element-update of resident_steps_kernel's step loop (ncu smsp__thread_inst_executed.sum of
-# one launch / (K * P * steps in the launch), captured on c2 and c1): the "algorithmic work" of the ALU roofline.
-NCU_RESIDENT_INSTR = {"source_sha256": "50003bae45ccf418daa7e0cf5905989b256153612eaa9679a289badc969e7cfb", "adamw": 51.50, "sgdm": 49.24}
+# one launch / (K * P * steps in the launch), captured on c2 and c1): the "algorithmic work" of the ALU roofline, which
+# is a bound on instruction issue.  The kernel uses packed fp32 instructions (two operations per lane each);
+# "scalar_equivalent" is the count of the same arithmetic issued one operation per instruction.
+NCU_RESIDENT_INSTR = {"source_sha256": "dbf5f9d72f3533f877a85fdd47f30eaa4c90e7f0f96090100f4c950e8d5f81a1", "adamw": 39.75, "sgdm": 40.73,
+                      "scalar_equivalent": {"adamw": 51.50, "sgdm": 49.24}}
 SM_COUNT, LANES_PER_SM_CLK = 148, 4 * 32      # 4 schedulers per SM, one warp instruction (32 lanes) each per clock
 
 
@@ -609,7 +612,9 @@ def run_resident(args, backend):
                      "unit": "G thread-instr/s", "frac": achieved / peak if achieved else None,
                      "peak_kind": f"{SM_COUNT} SMs x {LANES_PER_SM_CLK} lanes per clock x the median SM clock sampled "
                                   f"during the run ({sm_mhz:.0f} MHz)",
-                     "thread_instr_per_update": instr, "avg_launch_ms": total_ms / launches, "traffic": None},
+                     "thread_instr_per_update": instr,
+                     "scalar_equivalent_ops_per_update": NCU_RESIDENT_INSTR["scalar_equivalent"][w.opt] if instr else None,
+                     "avg_launch_ms": total_ms / launches, "traffic": None},
         "gpu_launches": int(launches), "clocks": clocks,
     }
     if clocks and clocks.get("sm_mhz"):

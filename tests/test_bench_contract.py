@@ -54,4 +54,5 @@ def test_recorded_instruction_counts_match_the_resident_kernel_source():
         "the resident-steps kernel changed since the ncu capture: re-capture and update NCU_RESIDENT_INSTR"
     # the ALU peak: 148 SMs x 4 schedulers x 32 lanes per clock
     assert bench.SM_COUNT * bench.LANES_PER_SM_CLK == 18944
-    assert 40 < bench.NCU_RESIDENT_INSTR["sgdm"] < bench.NCU_RESIDENT_INSTR["adamw"] < 60
+    assert 35 < bench.NCU_RESIDENT_INSTR["adamw"] < bench.NCU_RESIDENT_INSTR["sgdm"] < 45       # issued (packed fp32)
+    assert 45 < bench.NCU_RESIDENT_INSTR["scalar_equivalent"]["sgdm"] < bench.NCU_RESIDENT_INSTR["scalar_equivalent"]["adamw"] < 55
