@@ -305,6 +305,12 @@ int qsr_train_host(const qsr_config *cfg, const float *theta0_host, const float 
 int qsr_debug_box_muller(const uint32_t *words_dev, int64_t n, float *radius_dev, float *sin_dev, float *cos_dev,
                          void *cuda_stream);
 
+/* The two single-instruction special functions inside OPT of Eq. 1 as this library evaluates it (App. C.2's AdamW:
+ * the root of the second moment and the quotient m / denominator; the root also gives the Box-Muller radius):
+ * sqrt_dev[i] = sqrt.approx.ftz(x_dev[i]), rcp_dev[i] = rcp.approx.ftz(x_dev[i]) for n floats (device arrays, 4-byte
+ * aligned).  For tests that bound their error against binary64.  No context; one launch on cuda_stream; asynchronous. */
+int qsr_debug_fast_math(const float *x_dev, int64_t n, float *sqrt_dev, float *rcp_dev, void *cuda_stream);
+
 /* Text for a qsr_status. Never NULL. */
 const char *qsr_strerror(int status);
 

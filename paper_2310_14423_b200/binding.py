@@ -28,7 +28,7 @@ QSR_STATIC_SCRATCH_FLOATS = 1 << 20
 EXPORTS = ("qsr_config_check", "qsr_row_stride_hint", "qsr_config_learning_rate", "qsr_config_round_length", "qsr_config_schedule",
            "qsr_workspace_bytes", "qsr_init", "qsr_destroy", "qsr_round_length", "qsr_set_tensor_table", "qsr_clip_workspace_floats", "qsr_set_grad_clip", "qsr_set_params", "qsr_local_step",
            "qsr_local_step_sync", "qsr_parallel_step", "qsr_sync", "qsr_sync_sum_floats", "qsr_sync_partial", "qsr_local_step_partial", "qsr_sync_finish", "qsr_sync_static", "qsr_run", "qsr_launch_count",
-           "qsr_set_launch_shape", "qsr_set_graph_replay", "qsr_set_resident_steps", "qsr_train_host", "qsr_debug_box_muller", "qsr_strerror")
+           "qsr_set_launch_shape", "qsr_set_graph_replay", "qsr_set_resident_steps", "qsr_train_host", "qsr_debug_box_muller", "qsr_debug_fast_math", "qsr_strerror")
 
 
 class QsrConfig(C.Structure):
@@ -91,6 +91,7 @@ def lib():
             "qsr_set_resident_steps": (C.c_int, [vp, i32]),
             "qsr_train_host": (C.c_int, [cfg, vp, vp, vp, vp, vp, i64, i64, vp, vp, vp, i64, C.POINTER(i64), C.POINTER(i64)]),
             "qsr_debug_box_muller": (C.c_int, [vp, i64, vp, vp, vp, vp]),
+            "qsr_debug_fast_math": (C.c_int, [vp, i64, vp, vp, vp]),
             "qsr_strerror": (C.c_char_p, [C.c_int]),
         }
         for name in EXPORTS:
@@ -293,3 +294,9 @@ def qsr_debug_box_muller(words, radius, sine, cosine, stream: int = 0) -> None:
     n = int(words.numel())
     _check(lib().qsr_debug_box_muller(_dptr(words), n, _dptr(radius), _dptr(sine), _dptr(cosine), C.c_void_p(stream)),
            "qsr_debug_box_muller")
+
+
+def qsr_debug_fast_math(x, root, reciprocal, stream: int = 0) -> None:
+    """Test hook: the library's single-instruction square root and reciprocal of each float of x (CUDA tensors)."""
+    _check(lib().qsr_debug_fast_math(_dptr(x), int(x.numel()), _dptr(root), _dptr(reciprocal), C.c_void_p(stream)),
+           "qsr_debug_fast_math")

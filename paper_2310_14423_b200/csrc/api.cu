@@ -526,6 +526,16 @@ int qsr_debug_box_muller(const uint32_t *words_dev, int64_t n, float *radius_dev
     return cuda_rc(qsr::launch_box_muller_parts(words_dev, n, radius_dev, sin_dev, cos_dev, cuda_stream));
 }
 
+int qsr_debug_fast_math(const float *x_dev, int64_t n, float *sqrt_dev, float *rcp_dev, void *cuda_stream)
+{
+    if (n < 0) return QSR_EINVAL;
+    if (n == 0) return QSR_OK;
+    if (!x_dev || !sqrt_dev || !rcp_dev) return QSR_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(x_dev) | reinterpret_cast<uintptr_t>(sqrt_dev) | reinterpret_cast<uintptr_t>(rcp_dev)) & 3u)
+        return QSR_EALIGN;
+    return cuda_rc(qsr::launch_fast_math(x_dev, n, sqrt_dev, rcp_dev, cuda_stream));
+}
+
 int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
             int64_t *round_start, int64_t *round_len, int64_t cap, int64_t *n_rounds)
 {

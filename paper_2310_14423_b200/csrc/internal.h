@@ -112,6 +112,8 @@ int clip_grid(int64_t P);
 int launch_clip_coef(const StepParams &p, bool parallel, double max_norm, float *ws, const LaunchShape &shape, void *stream);
 // Test hook: radius, sine and cosine of the Box-Muller transform for n generator words (all device arrays).
 int launch_box_muller_parts(const uint32_t *words, int64_t n, float *radius, float *sine, float *cosine, void *stream);
+// Test hook: sqrt.approx.ftz and rcp.approx.ftz of n floats, as the optimizer update uses them.
+int launch_fast_math(const float *x, int64_t n, float *root, float *reciprocal, void *stream);
 // Both phases through the library's own static scratch; -1 if the sums exceed QSR_STATIC_SCRATCH_FLOATS, -2 if
 // `device` (the context's) is not the current device.
 int launch_sync_static(const SyncParams &p, const LaunchShape &shape, int device, void *stream);

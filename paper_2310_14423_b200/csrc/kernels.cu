@@ -836,6 +836,17 @@ __global__ void box_muller_parts_kernel(const uint32_t *words, int64_t n, float 
     }
 }
 
+// The two single-instruction special functions of the optimizer update (sqrt_fast for AdamW's root of the second
+// moment and the Box-Muller radius, rcp_fast for AdamW's quotient), for tests that bound their error.
+__global__ void fast_math_kernel(const float *x, int64_t n, float *root, float *reciprocal)
+{
+    const int64_t grid_stride = int64_t(gridDim.x) * blockDim.x;
+    for (int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += grid_stride) {
+        root[i] = sqrt_fast(x[i]);
+        reciprocal[i] = rcp_fast(x[i]);
+    }
+}
+
 // One thread per 16-byte column.  2^31 - 1 blocks of at least 64 threads cover rows of 2^39 floats, beyond any device
 // memory, so the kernels that rely on full coverage (local_step_kernel) never meet a capped grid.
 unsigned grid_for(int64_t P, int threads)
@@ -1027,6 +1038,15 @@ int launch_resident_steps(const ResidentParams &q, int opt, void *stream)
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (opt == QSR_OPT_SGDM) resident_steps_kernel<QSR_OPT_SGDM><<<unsigned(blocks), threads, smem, st>>>(q);
     else resident_steps_kernel<QSR_OPT_ADAMW><<<unsigned(blocks), threads, smem, st>>>(q);
+    return int(cudaGetLastError());
+}
+
+int launch_fast_math(const float *x, int64_t n, float *root, float *reciprocal, void *stream)
+{
+    int64_t blocks = (n + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks < 1) blocks = 1;
+    fast_math_kernel<<<unsigned(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(x, n, root, reciprocal);
     return int(cudaGetLastError());
 }
 

@@ -119,3 +119,26 @@ def test_argument_errors():
     assert L.qsr_debug_box_muller(None, 0, None, None, None, st) == B.QSR_OK
     torch.cuda.synchronize()
     assert not buf.any()
+
+
+def test_fast_square_root_and_reciprocal():
+    """The optimizer update's two special-function instructions against binary64: every fp32 mantissa (2^23 values) in
+    two binades each for the root (its error pattern repeats every two binades) and one for the reciprocal, plus the
+    ranges the path feeds them -- second moments down to 1e-30, denominators from eps = 1e-8 up."""
+    mant = np.arange(N_GRID, dtype=np.uint32)
+    parts = [(mant | np.uint32(0x3f800000)).view(np.float32),          # [1, 2)
+             (mant | np.uint32(0x40000000)).view(np.float32)]          # [2, 4)
+    rng = np.random.default_rng(4)
+    parts.append(np.exp(rng.uniform(np.log(1e-30), np.log(1e4), 1 << 22)).astype(np.float32))
+    x = np.concatenate(parts)
+    xd = torch.from_numpy(x).cuda()
+    root, rcp = torch.empty_like(xd), torch.empty_like(xd)
+    B.qsr_debug_fast_math(xd, root, rcp, stream=torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    x64 = x.astype(np.float64)
+    rel_root = root.cpu().numpy().astype(np.float64) / np.sqrt(x64) - 1
+    rel_rcp = rcp.cpu().numpy().astype(np.float64) * x64 - 1
+    print("sqrt.approx.ftz: max rel err %.3e, mean %.2e; rcp.approx.ftz: max %.3e, mean %.2e"
+          % (np.abs(rel_root).max(), rel_root.mean(), np.abs(rel_rcp).max(), rel_rcp.mean()))
+    assert np.abs(rel_root).max() <= 1.2e-7 and abs(rel_root.mean()) <= 2e-8
+    assert np.abs(rel_rcp).max() <= 1.6e-7 and abs(rel_rcp.mean()) <= 1e-8
