@@ -147,3 +147,33 @@ def test_argument_errors():
         assert e.value.status == B.QSR_ERANGE
     ctx.qsr_set_resident_steps(0)
     ctx.close()
+
+
+def test_packed_noise_equals_scalar_noise_bitwise():
+    """The resident launches evaluate the noise with packed fp32 instructions (two Box-Muller transforms per
+    instruction stream), the per-step kernel one lane at a time.  With eta = 1, lambda = 0, sigma = 1, no momentum and
+    no weight decay one SGD step from zero leaves theta = -z: 33.5 M normals (16.8 M words through the logarithm and
+    as many through the sine / cosine: most of the 2^23-point grid of each) must agree bit for bit."""
+    P, K, t = 1 << 22, 8, 12345
+    w = W.tiny_workload(W.OPT_SGDM, K=K, P=P, T=20000, sched=W.SCHED_CONST, eta_max=1.0, momentum=0.0,
+                        weight_decay=0.0, noise_std=1.0, rule=W.RULE_CONST_H, H_base=5)
+    zero = torch.zeros(P, device="cuda")
+    out = []
+    for resident in (0, 1):
+        theta = torch.zeros(K, P, device="cuda")
+        s1 = torch.zeros(K, P, device="cuda")
+        ctx = B.Context(B.make_config(w), theta, s1, None, zero, zero, stream=torch.cuda.current_stream().cuda_stream)
+        if resident:
+            ctx.qsr_set_resident_steps(1)
+            st, H = ctx.qsr_run(10000, 10001)          # a round of 5 from t = 10000: steps 10000 .. 10004 and a mean
+        else:
+            for u in range(10000, 10004):
+                ctx.qsr_local_step(u)
+            ctx.qsr_local_step_sync(10004, 10005)
+        torch.cuda.synchronize()
+        ctx.close()
+        out.append((theta, s1))
+    assert torch.equal(out[0][0], out[1][0]) and torch.equal(out[0][1], out[1][1])
+    # s1 holds the last step's gradient, i.e. that step's noise itself: not all the same, not all finite by accident
+    z = out[0][1]
+    assert bool(torch.isfinite(z).all()) and abs(float(z.mean())) < 1e-3 and abs(float(z.var()) - 1) < 1e-2
