@@ -222,3 +222,36 @@ def test_other_rules_and_schedules_equal_oracle():
     assert abs(100.0 * len(st) / cases[0].T - 13.2) <= 0.055      # step-decay table of App. G
     st, H = _same_schedule(cases[1])
     assert abs(100.0 * len(st) / cases[1].T - 14.4) <= 0.055
+
+
+def test_train_host_fails_before_touching_a_device_and_zeroes_its_outputs():
+    """Every check of qsr_train_host that can fail on the host comes before its first copy is enqueued, and the output
+    counters are zeroed at entry: bad arguments return their status with *launches = *n_rounds = 0 (no device needed;
+    on a machine without a GPU the valid call stops at the context's device query, QSR_ECUDA, also before any copy)."""
+    L = B.lib()
+    w = W.tiny_workload(W.OPT_ADAMW, K=2, P=64, T=10)
+    cfg = B.make_config(w)
+    host = np.zeros(64, np.float32)
+    ws_bytes = B.qsr_workspace_bytes(cfg)
+
+    def call(cfg_, workspace=4096, nbytes=ws_bytes, t_end=10, theta0=host):
+        n, launches = C.c_int64(77), C.c_int64(77)
+        st = np.empty(16, np.int64)
+        rc = L.qsr_train_host(C.byref(cfg_) if cfg_ is not None else None,
+                              theta0.ctypes.data if theta0 is not None else None, host.ctypes.data, host.ctypes.data,
+                              host.ctypes.data, workspace, nbytes, t_end, None, st.ctypes.data, st.ctypes.data, 16,
+                              C.byref(n), C.byref(launches))
+        return rc, n.value, launches.value
+
+    assert call(None) == (B.QSR_EINVAL, 0, 0)
+    assert call(cfg, theta0=None) == (B.QSR_EINVAL, 0, 0)
+    assert call(cfg, workspace=4096 + 16) == (B.QSR_EALIGN, 0, 0)          # workspace must be 256-byte aligned
+    assert call(cfg, nbytes=ws_bytes - 1) == (B.QSR_ERANGE, 0, 0)
+    assert call(cfg, t_end=11) == (B.QSR_ERANGE, 0, 0)
+    bad = B.make_config(w)
+    bad.K = 0
+    assert call(bad)[1:] == (0, 0) and call(bad)[0] < 0
+    import torch
+    if not torch.cuda.is_available():
+        # a valid call on a machine without a device: the context cannot be created, nothing was enqueued
+        assert call(cfg) == (B.QSR_ECUDA, 0, 0)
