@@ -46,7 +46,7 @@ L2_BYTES = 126e6
 # once, so traffic grows in proportion to K*P).  Valid only for the kernel source it was taken from: the hash covers
 # the noise generator, the optimizer update and local_step_kernel in csrc/kernels.cu.
 NCU_TRAFFIC = {
-    "step_source_sha256": "13c8e9bbf1a3e1513a8fe05499fb1a8af37d6dd6d63d0dd8179b671fd4e665fe",
+    "step_source_sha256": "35dba2222a898a7788bd1c2f05f600bec42d82d5b343b3587c17e1079241782c",
     "bytes_per_update": {"adamw": 24.07, "sgdm": 16.07},
 }
 

@@ -153,9 +153,15 @@ int qsr_set_tensor_table(qsr_ctx *ctx, int32_t n_tensors, const int64_t *tensor_
  * linear decay, off in the QSR runs), in the form of the paper's software: before OPT each worker's gradient is scaled
  * by min(1, max_norm / (||g||_2 + 1e-6)), the norm over all P coordinates of that worker (for qsr_parallel_step: of the
  * averaged gradient).  While it is on, every step launches two more kernels first: per-worker partial sums of g^2
- * (generated gradients are recomputed, not stored) and the K factors.  workspace_dev: caller-owned device memory of
- * qsr_clip_workspace_floats(ctx) floats, 16-byte aligned, borrowed until clipping is switched off or the context is
- * destroyed.  max_norm <= 0, infinite or NaN switches clipping off.  QSR_ERANGE if K exceeds 96. */
+ * (generated gradients are recomputed, not stored) and the K factors.  Inside qsr_run, where the library issues the
+ * steps of a round itself and nothing else touches the parameters in between, a plain step also computes its
+ * successor's partial sums from the new parameters it holds in registers, so only the first step of a round pays the
+ * norm pass (two launches per step instead of three, and no second read of the parameters); the factors are the same
+ * bits either way.  workspace_dev: caller-owned device memory of qsr_clip_workspace_floats(ctx) floats (one partial
+ * sum per worker and block of a step launch, so it grows with P: K * P / 256 + K floats), 16-byte aligned, borrowed
+ * until clipping is switched off or the context is destroyed.  max_norm <= 0, infinite or NaN switches clipping off.
+ * QSR_ERANGE if K exceeds 96.  The norm pass keeps K x (step threads) sums in shared memory: a step block size
+ * above 512 with K near 96 does not fit and makes the step return QSR_ECUDA. */
 int64_t qsr_clip_workspace_floats(const qsr_ctx *ctx);
 int qsr_set_grad_clip(qsr_ctx *ctx, double max_norm, float *workspace_dev);
 

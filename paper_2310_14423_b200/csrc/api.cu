@@ -113,15 +113,57 @@ struct RoundRange {
 };
 
 // With clipping on: enqueue the norm pass and the factor pass for this step and make the step kernel use the factors.
-int prepare_clip(qsr_ctx &x, qsr::StepParams &p, bool parallel)
+// `partials_ready`: the preceding step of the same round, launched by qsr_run, has already left this step's norm
+// partials in the workspace (Local OPT with generated gradients only), so only the factor pass is needed.
+int prepare_clip(qsr_ctx &x, qsr::StepParams &p, bool parallel, bool partials_ready = false)
 {
     if (!(x.clip_norm > 0.0)) return QSR_OK;
-    const int rows = parallel ? 1 : x.cfg.K;
-    const int grid = qsr::clip_grid(x.cfg.P);
-    x.launches += 2;
-    if (int err = qsr::launch_clip_coef(p, parallel, x.clip_norm, x.clip_ws, x.shape, x.stream)) return cuda_rc(err);
-    p.clip_coef = x.clip_ws + int64_t(grid) * rows;
+    if (parallel) {
+        x.launches += 2;
+        if (int err = qsr::launch_clip_coef_parallel(p, x.clip_norm, x.clip_ws, x.stream)) return cuda_rc(err);
+        p.clip_coef = x.clip_ws + qsr::clip_grid(x.cfg.P);
+        return QSR_OK;
+    }
+    const int64_t blocks = qsr::clip_norm_blocks(x.cfg.P, x.shape.step_threads);
+    if (!partials_ready) {
+        x.launches++;
+        if (int err = qsr::launch_clip_norms(p, x.clip_ws, x.shape, x.stream)) return cuda_rc(err);
+    }
+    x.launches++;
+    if (int err = qsr::launch_clip_factors(x.clip_ws, blocks, x.cfg.K, x.clip_norm, x.stream)) return cuda_rc(err);
+    p.clip_coef = x.clip_ws + blocks * x.cfg.K;
     return QSR_OK;
+}
+
+// Inside a round qsr_run issues every step itself and nothing else touches the parameters in between, so with
+// clipping on a plain step can compute its successor's gradient norms on the side (the new parameters are in its
+// registers) and the successor skips its norm pass.  Needs room for K x threads sums next to the step's ring.
+// A step that also evaluates the next step's noise is bound by its instruction stream rather than by the bytes it
+// keeps in flight, and gains more from a third or fourth resident block than from a deep ring: at most four rows in
+// flight (ViT-B/16 shape, K = 16: 6.24 ms per step with eight, 5.84 with four; the block size stays, because the norm
+// partials are laid out per block of the step).
+qsr::LaunchShape clip_fold_shape(const qsr_ctx &x)
+{
+    qsr::LaunchShape s = x.shape;
+    if (s.step_rows == 0 || s.step_rows > 4) s.step_rows = 4;
+    return s;
+}
+
+bool clip_fold_applies(const qsr_ctx &x)
+{
+    if (!(x.clip_norm > 0.0)) return false;
+    const qsr::LaunchShape s = clip_fold_shape(x);
+    return qsr::step_shared_bytes(x.cfg.opt, false, s.step_rows, s.step_threads, x.cfg.K) <= size_t(227) * 1024;
+}
+
+// A plain local step of qsr_run's own loop (generated gradients).
+int run_local_step(qsr_ctx &x, int64_t t, bool partials_ready, bool leave_next_partials)
+{
+    qsr::StepParams p = step_params(x, t, nullptr);
+    if (int rc = prepare_clip(x, p, false, partials_ready)) return rc;
+    if (leave_next_partials) p.norm_partial = x.clip_ws;
+    x.launches++;
+    return cuda_rc(qsr::launch_step(p, x.cfg.opt, leave_next_partials ? clip_fold_shape(x) : x.shape, x.stream));
 }
 
 constexpr size_t kMaxCachedGraphs = 48;
@@ -385,8 +427,11 @@ int qsr_set_tensor_table(qsr_ctx *ctx, int32_t n_tensors, const int64_t *tensor_
 int64_t qsr_clip_workspace_floats(const qsr_ctx *ctx)
 {
     if (!ctx) return QSR_EINVAL;
-    // partials [norm grid, K] followed by the K factors; the grid never exceeds kNormGrid whatever the block size
-    return round_up4(int64_t(qsr::kNormGrid) * ctx->cfg.K + ctx->cfg.K);
+    // Local OPT: partials [blocks of a step launch, K] followed by the K factors; the smallest block (64 threads) gives
+    // the most blocks.  Algorithm 1: at most kNormGrid partials and one factor.
+    const int64_t local = qsr::clip_norm_blocks(ctx->cfg.P, 64) * ctx->cfg.K + ctx->cfg.K;
+    const int64_t parallel = int64_t(qsr::kNormGrid) + 1;
+    return round_up4(local > parallel ? local : parallel);
 }
 
 int qsr_set_grad_clip(qsr_ctx *ctx, double max_norm, float *workspace_dev)
@@ -398,7 +443,7 @@ int qsr_set_grad_clip(qsr_ctx *ctx, double max_norm, float *workspace_dev)
     }
     if (!workspace_dev) return QSR_EINVAL;
     if (!aligned16(workspace_dev)) return QSR_EALIGN;
-    if (ctx->cfg.K > 96) return QSR_ERANGE;   // the norm pass keeps K x kNormThreads running sums in 48 KB of shared memory
+    if (ctx->cfg.K > qsr::kMaxClipK) return QSR_ERANGE;   // the norm pass keeps K x (step threads) sums in shared memory
     ctx->clip_norm = max_norm; ctx->clip_ws = workspace_dev;
     return QSR_OK;
 }
@@ -415,21 +460,27 @@ int qsr_parallel_step(qsr_ctx *ctx, int64_t t, const float *grads)
     return cuda_rc(qsr::launch_parallel_step(p, ctx->cfg.opt, ctx->shape, ctx->stream));
 }
 
-int qsr_local_step_sync(qsr_ctx *ctx, int64_t t, const float *grads, int64_t t_next)
+// The round's last step and its synchronization.  `partials_ready` as in prepare_clip (qsr_run only).
+static int local_step_sync_impl(qsr_ctx *ctx, int64_t t, const float *grads, int64_t t_next, bool partials_ready)
 {
     if (!ctx) return QSR_EINVAL;
     if (t < 0 || t >= ctx->cfg.T || t < ctx->t_state_origin || t_next < 0 || t_next > ctx->cfg.T) return QSR_ERANGE;
-    if (ctx->cfg.state_sync != QSR_STATE_KEEP) {
-        // Averaging or resetting the optimizer state needs the stand-alone kernel: two launches.
-        if (int rc = qsr_local_step(ctx, t, grads)) return rc;
-        return qsr_sync(ctx, t_next);
-    }
     if (!grads && !ctx->lambda) return QSR_EINVAL;
     if (!aligned16(grads)) return QSR_EALIGN;
     qsr::StepParams p = step_params(*ctx, t, grads);
-    if (int rc = prepare_clip(*ctx, p, false)) return rc;
+    if (int rc = prepare_clip(*ctx, p, false, partials_ready)) return rc;
     ctx->launches++;
+    if (ctx->cfg.state_sync != QSR_STATE_KEEP) {
+        // Averaging or resetting the optimizer state needs the stand-alone kernel: a plain step, then the sync.
+        if (int rc = cuda_rc(qsr::launch_step(p, ctx->cfg.opt, ctx->shape, ctx->stream))) return rc;
+        return qsr_sync(ctx, t_next);
+    }
     return cuda_rc(qsr::launch_step_mean(p, ctx->cfg.opt, ctx->shape, ctx->stream));
+}
+
+int qsr_local_step_sync(qsr_ctx *ctx, int64_t t, const float *grads, int64_t t_next)
+{
+    return local_step_sync_impl(ctx, t, grads, t_next, false);
 }
 
 int qsr_sync(qsr_ctx *ctx, int64_t t_next)
@@ -563,11 +614,16 @@ int qsr_run(qsr_ctx *ctx, int64_t t_begin, int64_t t_end,
                 h += n_plain + (fused ? 1 : 0);
             }
         }
-        for (; h + 1 < H; ++h)
-            if (int rc = qsr_local_step(ctx, t + h, nullptr)) return rc;
+        // with clipping on, each plain step leaves its successor's gradient-norm partials behind (clip_fold_applies)
+        const bool fold = h == 0 && clip_fold_applies(*ctx);
+        bool partials_ready = false;
+        for (; h + 1 < H; ++h) {
+            if (int rc = run_local_step(*ctx, t + h, partials_ready, fold)) return rc;
+            partials_ready = fold;
+        }
         // the round's last step and the parameter averaging, in one launch when the state is kept per worker
         if (h < H)
-            if (int rc = qsr_local_step_sync(ctx, t + H - 1, nullptr, t + H)) return rc;
+            if (int rc = local_step_sync_impl(ctx, t + H - 1, nullptr, t + H, partials_ready)) return rc;
         if (s < cap) {
             round_start[s] = t;
             round_len[s] = H;

@@ -38,10 +38,12 @@ struct StepParams {
     const float *wd_scale;         // device [n_tensors]: factor on the weight decay of each tensor
     const float *clip_coef;        // NULL, or device [K] ([1] for Algorithm 1): gradient-clipping factor per worker
     float *sum_out;                // step fused with the partial sums of a sharded synchronization: device [P4]
+    float *norm_partial;           // not NULL: the step also leaves the NEXT step's gradient-norm partials here
 };
 
-constexpr int kNormGrid = 1184;    // blocks of the gradient-norm pass (8 per SM on a 148-SM part)
-constexpr int kNormThreads = 128;  // its block size: K x 128 running sums must fit 48 KB of shared memory (K <= 96)
+constexpr int kNormGrid = 1184;    // blocks of Algorithm 1's gradient-norm pass (8 per SM on a 148-SM part)
+constexpr int kNormThreads = 128;  // its block size
+constexpr int kMaxClipK = 96;      // Local OPT's norm pass keeps K x threads sums in shared memory
 
 struct SyncParams {
     float *slab[3];           // arrays to average (theta first), then arrays to zero
@@ -107,9 +109,16 @@ int launch_sync_finish(const SyncParams &p, const LaunchShape &shape, void *stre
 inline int sync_launches(const SyncParams &p) { return p.n_zero > 0 ? 2 : 1; }       // of launch_sync / launch_sync_finish
 int launch_broadcast(float *theta, const float *theta0, int64_t P, int64_t stride, int32_t K,
                      const LaunchShape &shape, void *stream);
-// Gradient clipping: grid of the norm pass and the two passes that leave the factors at ws + clip_grid(...) * rows.
+// Gradient clipping.  Local OPT: the norm pass writes clip_norm_blocks(P, step threads) x K partial sums to ws (a step
+// launched with StepParams::norm_partial set leaves the same numbers for its successor), the factor pass turns them
+// into K factors at ws + blocks * K.  Algorithm 1: both passes at once, the factor at ws + clip_grid(P).
 int clip_grid(int64_t P);
-int launch_clip_coef(const StepParams &p, bool parallel, double max_norm, float *ws, const LaunchShape &shape, void *stream);
+int64_t clip_norm_blocks(int64_t P, int threads);
+int launch_clip_norms(const StepParams &p, float *ws, const LaunchShape &shape, void *stream);
+int launch_clip_factors(float *ws, int64_t blocks, int rows, double max_norm, void *stream);
+int launch_clip_coef_parallel(const StepParams &p, double max_norm, float *ws, void *stream);
+// Dynamic shared memory of a step launch (the ring, plus next_norm_rows x threads floats).
+size_t step_shared_bytes(int opt, bool ext_grad, int stages, int threads, int next_norm_rows);
 // Test hook: radius, sine and cosine of the Box-Muller transform for n generator words (all device arrays).
 int launch_box_muller_parts(const uint32_t *words, int64_t n, float *radius, float *sine, float *cosine, void *stream);
 // Test hook: sqrt.approx.ftz and rcp.approx.ftz of n floats, as the optimizer update uses them.

@@ -192,167 +192,9 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait_all_but() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// One local step of all K workers.
-//
-// Memory pipeline.  A thread owns one 16-byte column and walks down the K rows.  Row k's operands (theta, state1,
-// [state2], [gradient]) are fetched by cp.async into the thread's private slots of a STAGES-deep ring in shared
-// memory; the ring is filled STAGES rows ahead, and as soon as a row has been copied to registers its slot is
-// refilled with row k + STAGES.  With 256 threads, 8 stages and AdamW's three operands a CTA holds 96 KB of loads in
-// flight (two CTAs per SM), against about 60 KB per SM when the rows in flight had to live in registers; on B200
-// that took the sustained ViT-B/16-shaped AdamW step from 5.6 ms to 5.35 ms, and trimming the instruction stream
-// (see the noise section) brought it to 5.3 ms, 97-98 % of the rate of a device-to-device copy.
-// Results go straight from registers to global memory with 128-bit stores.
-//
-// Round end.  With FUSE != 0 the step is the last of its round and the kernel also ends the round (Algorithm 2's
-// averaging, state kept per worker): the thread that owns a column sees every worker's new parameters anyway, so it
-// sums them as it goes (k ascending, fp32: the order of the stand-alone sync kernel, hence the same bits).
-// FUSE_MEAN writes the mean to all K rows instead of the K different values: the averaging then costs no HBM traffic
-// at all, theta is read once and written once exactly as in a plain step.  FUSE_SUM is the multi-GPU form: the
-// column's sum goes to p.sum_out (the buffer that is all-reduced over processes) and theta is not written at all,
-// since the finish kernel will overwrite every row with the global mean.
-//
-// EXTRAS selects the build that honours the per-tensor weight-decay table and the clipping factors; the plain build
-// (no table, clipping off: every run of the paper's QSR experiments) does not carry their tests in the row loop.
-
-template <int OPT, bool EXT_GRAD>
-struct StepOperands {
-    static constexpr int kStateSlabs = OPT == QSR_OPT_ADAMW ? 2 : 1;
-    static constexpr int kCount = 1 + kStateSlabs + (EXT_GRAD ? 1 : 0);   // slots per row and thread
-};
-
-template <int OPT, bool EXT_GRAD, int STAGES, int FUSE, bool EXTRAS>
-__global__ void local_step_kernel(const __grid_constant__ StepParams p)
-{
-    extern __shared__ float4 ring[];   // [STAGES][operands][blockDim.x]
-    constexpr int NOP = StepOperands<OPT, EXT_GRAD>::kCount;
-    const int tid = threadIdx.x, bd = blockDim.x;
-    const int64_t n_col = (p.P + 3) >> 2;
-    const int64_t j = int64_t(blockIdx.x) * bd + tid;      // the grid has one thread per column (see grid_for)
-    if (j >= n_col) return;
-    {
-        const int64_t i0 = j << 2;
-        const float wdv = EXTRAS ? weight_decay_at<OPT>(p, i0) : (OPT == QSR_OPT_SGDM ? p.wd : p.eta_wd);
-        if (i0 + 4 <= p.P) {
-            float4 lam = make_float4(0.f, 0.f, 0.f, 0.f), ths = lam;
-            if (!EXT_GRAD) {
-                lam = ld4(p.lambda + i0);
-                ths = ld4(p.theta_star + i0);
-            }
-            auto fetch = [&](int k, int stage) {
-                const int64_t e = int64_t(k) * p.stride + i0;
-                float4 *slot = ring + (stage * NOP) * bd + tid;
-                cp_async16(slot, p.theta + e);
-                cp_async16(slot + bd, p.s1 + e);
-                if (OPT == QSR_OPT_ADAMW) cp_async16(slot + 2 * bd, p.s2 + e);
-                if (EXT_GRAD) cp_async16(slot + (NOP - 1) * bd, p.grads + e);
-            };
-#pragma unroll
-            for (int s = 0; s < STAGES; ++s) {      // fill the ring; one group per row, empty groups keep the count uniform
-                if (s < p.K) fetch(s, s);
-                cp_async_commit();
-            }
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            int stage = 0;
-            for (int k = 0; k < p.K; ++k) {
-                cp_async_wait_all_but<STAGES - 1>();                 // row k has landed
-                const float4 *slot = ring + (stage * NOP) * bd + tid;
-                float4 th = slot[0], a = slot[bd], b = make_float4(0.f, 0.f, 0.f, 0.f), g;
-                if (OPT == QSR_OPT_ADAMW) b = slot[2 * bd];
-                if (EXT_GRAD) g = slot[(NOP - 1) * bd];
-                if (k + STAGES < p.K) fetch(k + STAGES, stage);      // the slot is free again: refill it
-                cp_async_commit();
-                stage = stage + 1 == STAGES ? 0 : stage + 1;
-                if (!EXT_GRAD) {
-                    const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.round_key);
-                    g.x = fmaf(p.sigma, z.x, lam.x * (th.x - ths.x));
-                    g.y = fmaf(p.sigma, z.y, lam.y * (th.y - ths.y));
-                    g.z = fmaf(p.sigma, z.z, lam.z * (th.z - ths.z));
-                    g.w = fmaf(p.sigma, z.w, lam.w * (th.w - ths.w));
-                }
-                if (EXTRAS && p.clip_coef) {   // gradient clipping: this worker's factor min(1, c / (||g|| + 1e-6))
-                    const float cs = __ldg(p.clip_coef + k);
-                    g.x *= cs; g.y *= cs; g.z *= cs; g.w *= cs;
-                }
-                opt_update<OPT>(th.x, a.x, b.x, g.x, p, wdv);
-                opt_update<OPT>(th.y, a.y, b.y, g.y, p, wdv);
-                opt_update<OPT>(th.z, a.z, b.z, g.z, p, wdv);
-                opt_update<OPT>(th.w, a.w, b.w, g.w, p, wdv);
-                const int64_t e = int64_t(k) * p.stride + i0;
-                if (FUSE != FUSE_NONE) acc = add4(acc, th);
-                else st4(p.theta + e, th);
-                st4(p.s1 + e, a);
-                if (OPT == QSR_OPT_ADAMW) st4(p.s2 + e, b);
-            }
-            if (FUSE == FUSE_MEAN) {
-                // At the power-capped clock the SGD step is close to issue-bound and every instruction of this
-                // epilogue shows (the round-end launch ran 7.5 % more instructions than a plain step and took 4-6 %
-                // longer on boxes that hold only 1.46 GHz): for K a power of two -- every run configuration -- 1/K is
-                // exact and the product equals the quotient bit for bit, and the row pointer advances by addition.
-                const float4 mean = (p.K & (p.K - 1)) == 0
-                                        ? make_float4(acc.x * p.inv_K, acc.y * p.inv_K, acc.z * p.inv_K, acc.w * p.inv_K)
-                                        : div4(acc, float(p.K));
-                float *row = p.theta + i0;
-#pragma unroll 4
-                for (int k = 0; k < p.K; ++k) {
-                    st4(row, mean);
-                    row += p.stride;
-                }
-            } else if (FUSE == FUSE_SUM) {
-                st4(p.sum_out + i0, acc);
-            }
-        } else {
-            // Ragged last column: P is not a multiple of 4.  Scalar accesses, nothing beyond P is touched.
-            for (int64_t i = i0; i < p.P; ++i) {
-                const int c = int(i - i0);                                  // 0, 1 or 2
-                float acc = 0.f;
-                for (int k = 0; k < p.K; ++k) {
-                    const int64_t e = int64_t(k) * p.stride + i;
-                    float th = p.theta[e], a = p.s1[e], b = OPT == QSR_OPT_ADAMW ? p.s2[e] : 0.f;
-                    float g;
-                    if (EXT_GRAD) {
-                        g = p.grads[e];
-                    } else {
-                        const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.round_key);
-                        const float zc = c == 0 ? z.x : (c == 1 ? z.y : z.z);
-                        g = fmaf(p.sigma, zc, p.lambda[i] * (th - p.theta_star[i]));
-                    }
-                    if (EXTRAS && p.clip_coef) g *= __ldg(p.clip_coef + k);
-                    opt_update<OPT>(th, a, b, g, p, wdv);
-                    if (FUSE != FUSE_NONE) acc += th;
-                    else p.theta[e] = th;
-                    p.s1[e] = a;
-                    if (OPT == QSR_OPT_ADAMW) p.s2[e] = b;
-                }
-                if (FUSE == FUSE_MEAN) {
-                    const float mean = acc / float(p.K);
-                    for (int k = 0; k < p.K; ++k) p.theta[int64_t(k) * p.stride + i] = mean;
-                } else if (FUSE == FUSE_SUM) {
-                    p.sum_out[i] = acc;
-                }
-            }
-        }
-    }
-}
-
-// Sum over rows of one 16-byte column, k ascending, eight loads in flight.
-__device__ __forceinline__ float4 column_sum(const float *slab, int64_t i0, int64_t stride, int K)
-{
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    int k = 0;
-    for (; k + 8 <= K; k += 8) {
-        float4 v[8];
-#pragma unroll
-        for (int r = 0; r < 8; ++r) v[r] = ld4(slab + int64_t(k + r) * stride + i0);
-#pragma unroll
-        for (int r = 0; r < 8; ++r) acc = add4(acc, v[r]);
-    }
-    for (; k < K; ++k) acc = add4(acc, ld4(slab + int64_t(k) * stride + i0));
-    return acc;
-}
-
 // ---------------------------------------------------------------------------------------------- packed arithmetic
 //
-// The kernels below this point that are bound by instruction issue rather than by memory -- Algorithm 1's step, the
+// The kernels that are bound by instruction issue rather than by memory -- Algorithm 1's step, the
 // gradient-norm pass of clipping and the register-resident launches -- evaluate the noise, the gradient and the
 // optimizer update two lanes at a time.  Every component is rounded exactly like its scalar form, so the results are
 // the bits of noise4 / opt_update (the tests that compare these kernels with the per-step kernel bit for bit cover it).
@@ -476,6 +318,220 @@ __device__ __forceinline__ void opt_update4(float4 &th, float4 &a, float4 &b, fl
     b = make_float4(b0.x, b0.y, b1.x, b1.y);
 }
 
+// 16-byte load when the whole column lies inside the row, scalar loads (zeros beyond P) for the ragged last column.
+__device__ __forceinline__ float4 ld4_guarded(const float *q, int valid)
+{
+    if (valid == 4) return ld4(q);
+    return make_float4(q[0], valid > 1 ? q[1] : 0.f, valid > 2 ? q[2] : 0.f, 0.f);
+}
+
+// Sum of squares of worker k's generated gradient over the (up to four) coordinates of column j at step `step`, the
+// parameters given in th: what the global norm of gradient clipping (App. C.2) is made of.  One definition for the
+// norm pass and for the step kernel that computes the next step's norms on the side, so that both give the same bits.
+__device__ __forceinline__ float column_sq(const StepParams &p, int64_t j, uint32_t step, int k, float4 th, float4 lam,
+                                           float4 ths, int valid)
+{
+    const float4 z = noise4_packed(j, step, p.worker0 + uint32_t(k), p.round_key);
+    float4 g = gradient4(p.sigma, z, lam, th, ths);
+    if (valid < 4) {                   // ragged last column: the lanes beyond P do not count
+        g.y = valid > 1 ? g.y : 0.f;
+        g.z = valid > 2 ? g.z : 0.f;
+        g.w = 0.f;
+    }
+    return fmaf(g.x, g.x, g.y * g.y) + fmaf(g.z, g.z, g.w * g.w);
+}
+
+// Block reduction of per-thread values acc[row][thread] to partial[block][row]: warp w folds rows w, w + n_warps, ...
+// in a fixed order (lanes stride over the threads, then a butterfly), so the result does not depend on timing.
+__device__ __forceinline__ void reduce_rows_to_partials(const float *acc, int rows, float *partial)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    for (int r = warp; r < rows; r += n_warps) {
+        float v = 0.f;
+        for (int t = lane; t < int(blockDim.x); t += 32) v += acc[r * blockDim.x + t];
+        for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) partial[int64_t(blockIdx.x) * rows + r] = v;
+    }
+}
+
+// One local step of all K workers.
+//
+// Memory pipeline.  A thread owns one 16-byte column and walks down the K rows.  Row k's operands (theta, state1,
+// [state2], [gradient]) are fetched by cp.async into the thread's private slots of a STAGES-deep ring in shared
+// memory; the ring is filled STAGES rows ahead, and as soon as a row has been copied to registers its slot is
+// refilled with row k + STAGES.  With 256 threads, 8 stages and AdamW's three operands a CTA holds 96 KB of loads in
+// flight (two CTAs per SM), against about 60 KB per SM when the rows in flight had to live in registers; on B200
+// that took the sustained ViT-B/16-shaped AdamW step from 5.6 ms to 5.35 ms, and trimming the instruction stream
+// (see the noise section) brought it to 5.3 ms, 97-98 % of the rate of a device-to-device copy.
+// Results go straight from registers to global memory with 128-bit stores.
+//
+// Round end.  With FUSE != 0 the step is the last of its round and the kernel also ends the round (Algorithm 2's
+// averaging, state kept per worker): the thread that owns a column sees every worker's new parameters anyway, so it
+// sums them as it goes (k ascending, fp32: the order of the stand-alone sync kernel, hence the same bits).
+// FUSE_MEAN writes the mean to all K rows instead of the K different values: the averaging then costs no HBM traffic
+// at all, theta is read once and written once exactly as in a plain step.  FUSE_SUM is the multi-GPU form: the
+// column's sum goes to p.sum_out (the buffer that is all-reduced over processes) and theta is not written at all,
+// since the finish kernel will overwrite every row with the global mean.
+//
+// EXTRAS selects the build that honours the per-tensor weight-decay table and the clipping factors; the plain build
+// (no table, clipping off: every run of the paper's QSR experiments) does not carry their tests in the row loop.
+
+template <int OPT, bool EXT_GRAD>
+struct StepOperands {
+    static constexpr int kStateSlabs = OPT == QSR_OPT_ADAMW ? 2 : 1;
+    static constexpr int kCount = 1 + kStateSlabs + (EXT_GRAD ? 1 : 0);   // slots per row and thread
+};
+
+// NEXTNORM (gradient clipping on, gradients generated, plain step): the thread that has just formed a worker's new
+// parameters also evaluates that worker's NEXT gradient on them and leaves its sum of squares in shared memory; the
+// block folds the K x blockDim values into p.norm_partial, laid out and summed exactly as the stand-alone norm pass
+// (column_sqnorm_kernel) does.  The following step then needs no norm pass of its own: the parameters are not read a
+// second time, and the extra noise evaluation runs in issue slots the memory-bound step leaves free.
+template <int OPT, bool EXT_GRAD, int STAGES, int FUSE, bool EXTRAS, bool NEXTNORM>
+__global__ void local_step_kernel(const __grid_constant__ StepParams p)
+{
+    extern __shared__ float4 ring[];   // [STAGES][operands][blockDim.x], then (NEXTNORM) float [K][blockDim.x]
+    constexpr int NOP = StepOperands<OPT, EXT_GRAD>::kCount;
+    const int tid = threadIdx.x, bd = blockDim.x;
+    const int64_t n_col = (p.P + 3) >> 2;
+    const int64_t j = int64_t(blockIdx.x) * bd + tid;      // the grid has one thread per column (see grid_for)
+    float *norm_acc = reinterpret_cast<float *>(ring + STAGES * NOP * bd);
+    if (j >= n_col) {
+        if (!NEXTNORM) return;
+        for (int k = 0; k < p.K; ++k) norm_acc[k * bd + tid] = 0.f;     // stays for the block's reduction below
+    } else {
+        const int64_t i0 = j << 2;
+        const float wdv = EXTRAS ? weight_decay_at<OPT>(p, i0) : (OPT == QSR_OPT_SGDM ? p.wd : p.eta_wd);
+        if (i0 + 4 <= p.P) {
+            float4 lam = make_float4(0.f, 0.f, 0.f, 0.f), ths = lam;
+            if (!EXT_GRAD) {
+                lam = ld4(p.lambda + i0);
+                ths = ld4(p.theta_star + i0);
+            }
+            auto fetch = [&](int k, int stage) {
+                const int64_t e = int64_t(k) * p.stride + i0;
+                float4 *slot = ring + (stage * NOP) * bd + tid;
+                cp_async16(slot, p.theta + e);
+                cp_async16(slot + bd, p.s1 + e);
+                if (OPT == QSR_OPT_ADAMW) cp_async16(slot + 2 * bd, p.s2 + e);
+                if (EXT_GRAD) cp_async16(slot + (NOP - 1) * bd, p.grads + e);
+            };
+#pragma unroll
+            for (int s = 0; s < STAGES; ++s) {      // fill the ring; one group per row, empty groups keep the count uniform
+                if (s < p.K) fetch(s, s);
+                cp_async_commit();
+            }
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            int stage = 0;
+            for (int k = 0; k < p.K; ++k) {
+                cp_async_wait_all_but<STAGES - 1>();                 // row k has landed
+                const float4 *slot = ring + (stage * NOP) * bd + tid;
+                float4 th = slot[0], a = slot[bd], b = make_float4(0.f, 0.f, 0.f, 0.f), g;
+                if (OPT == QSR_OPT_ADAMW) b = slot[2 * bd];
+                if (EXT_GRAD) g = slot[(NOP - 1) * bd];
+                if (k + STAGES < p.K) fetch(k + STAGES, stage);      // the slot is free again: refill it
+                cp_async_commit();
+                stage = stage + 1 == STAGES ? 0 : stage + 1;
+                if (!EXT_GRAD) {
+                    const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.round_key);
+                    g.x = fmaf(p.sigma, z.x, lam.x * (th.x - ths.x));
+                    g.y = fmaf(p.sigma, z.y, lam.y * (th.y - ths.y));
+                    g.z = fmaf(p.sigma, z.z, lam.z * (th.z - ths.z));
+                    g.w = fmaf(p.sigma, z.w, lam.w * (th.w - ths.w));
+                }
+                if (EXTRAS && p.clip_coef) {   // gradient clipping: this worker's factor min(1, c / (||g|| + 1e-6))
+                    const float cs = __ldg(p.clip_coef + k);
+                    g.x *= cs; g.y *= cs; g.z *= cs; g.w *= cs;
+                }
+                opt_update<OPT>(th.x, a.x, b.x, g.x, p, wdv);
+                opt_update<OPT>(th.y, a.y, b.y, g.y, p, wdv);
+                opt_update<OPT>(th.z, a.z, b.z, g.z, p, wdv);
+                opt_update<OPT>(th.w, a.w, b.w, g.w, p, wdv);
+                const int64_t e = int64_t(k) * p.stride + i0;
+                if (FUSE != FUSE_NONE) acc = add4(acc, th);
+                else st4(p.theta + e, th);
+                st4(p.s1 + e, a);
+                if (OPT == QSR_OPT_ADAMW) st4(p.s2 + e, b);
+                if (NEXTNORM) norm_acc[k * bd + tid] = column_sq(p, j, p.step + 1u, k, th, lam, ths, 4);
+            }
+            if (FUSE == FUSE_MEAN) {
+                // At the power-capped clock the SGD step is close to issue-bound and every instruction of this
+                // epilogue shows (the round-end launch ran 7.5 % more instructions than a plain step and took 4-6 %
+                // longer on boxes that hold only 1.46 GHz): for K a power of two -- every run configuration -- 1/K is
+                // exact and the product equals the quotient bit for bit, and the row pointer advances by addition.
+                const float4 mean = (p.K & (p.K - 1)) == 0
+                                        ? make_float4(acc.x * p.inv_K, acc.y * p.inv_K, acc.z * p.inv_K, acc.w * p.inv_K)
+                                        : div4(acc, float(p.K));
+                float *row = p.theta + i0;
+#pragma unroll 4
+                for (int k = 0; k < p.K; ++k) {
+                    st4(row, mean);
+                    row += p.stride;
+                }
+            } else if (FUSE == FUSE_SUM) {
+                st4(p.sum_out + i0, acc);
+            }
+        } else {
+            // Ragged last column: P is not a multiple of 4.  Scalar accesses, nothing beyond P is touched.
+            for (int64_t i = i0; i < p.P; ++i) {
+                const int c = int(i - i0);                                  // 0, 1 or 2
+                float acc = 0.f;
+                for (int k = 0; k < p.K; ++k) {
+                    const int64_t e = int64_t(k) * p.stride + i;
+                    float th = p.theta[e], a = p.s1[e], b = OPT == QSR_OPT_ADAMW ? p.s2[e] : 0.f;
+                    float g;
+                    if (EXT_GRAD) {
+                        g = p.grads[e];
+                    } else {
+                        const float4 z = noise4(j, p.step, p.worker0 + uint32_t(k), p.round_key);
+                        const float zc = c == 0 ? z.x : (c == 1 ? z.y : z.z);
+                        g = fmaf(p.sigma, zc, p.lambda[i] * (th - p.theta_star[i]));
+                    }
+                    if (EXTRAS && p.clip_coef) g *= __ldg(p.clip_coef + k);
+                    opt_update<OPT>(th, a, b, g, p, wdv);
+                    if (FUSE != FUSE_NONE) acc += th;
+                    else p.theta[e] = th;
+                    p.s1[e] = a;
+                    if (OPT == QSR_OPT_ADAMW) p.s2[e] = b;
+                }
+                if (FUSE == FUSE_MEAN) {
+                    const float mean = acc / float(p.K);
+                    for (int k = 0; k < p.K; ++k) p.theta[int64_t(k) * p.stride + i] = mean;
+                } else if (FUSE == FUSE_SUM) {
+                    p.sum_out[i] = acc;
+                }
+            }
+            if (NEXTNORM) {            // the ragged column's share of the next norms, from the values just written
+                const int valid = int(p.P - i0);
+                const float4 lam = ld4_guarded(p.lambda + i0, valid), ths = ld4_guarded(p.theta_star + i0, valid);
+                for (int k = 0; k < p.K; ++k)
+                    norm_acc[k * bd + tid] = column_sq(p, j, p.step + 1u, k, ld4_guarded(p.theta + int64_t(k) * p.stride + i0, valid),
+                                                       lam, ths, valid);
+            }
+        }
+    }
+    if (NEXTNORM) {
+        __syncthreads();
+        reduce_rows_to_partials(norm_acc, p.K, p.norm_partial);
+    }
+}
+
+// Sum over rows of one 16-byte column, k ascending, eight loads in flight.
+__device__ __forceinline__ float4 column_sum(const float *slab, int64_t i0, int64_t stride, int K)
+{
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    int k = 0;
+    for (; k + 8 <= K; k += 8) {
+        float4 v[8];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) v[r] = ld4(slab + int64_t(k + r) * stride + i0);
+#pragma unroll
+        for (int r = 0; r < 8; ++r) acc = add4(acc, v[r]);
+    }
+    for (; k < K; ++k) acc = add4(acc, ld4(slab + int64_t(k) * stride + i0));
+    return acc;
+}
+
 // ---------------------------------------------------------------------------------------------- Algorithm 1
 
 // Parallel OPT: the single model lives in row 0 of the slabs; the K workers' gradients are all taken at that one
@@ -546,44 +602,73 @@ __global__ void parallel_step_kernel(const __grid_constant__ StepParams p)
 
 // ---------------------------------------------------------------------------------------------- gradient clipping
 
-// 16-byte load when the whole column lies inside the row, scalar loads (zeros beyond P) for the ragged last column.
-__device__ __forceinline__ float4 ld4_guarded(const float *q, int valid)
+// Pass 1 of global-norm clipping (App. C.2) for Local OPT: per worker k the sum of squares of the gradient its step
+// will use, as partial sums per block.  Generated gradients are recomputed here with the very expressions of the step
+// kernel -- the noise is a pure function of (seed, worker, step, coordinate) -- so nothing has to be stored: the pass
+// reads theta once (4 B per update).  The geometry is the step kernel's (one thread per column, the step's block
+// size) and the per-column value and the block's reduction are shared code, so the partials equal, bit for bit, what a
+// step launched with NEXTNORM leaves behind for its successor.  partial is [gridDim.x, K].
+template <bool EXT_GRAD>
+__global__ void column_sqnorm_kernel(const __grid_constant__ StepParams p, float *partial)
 {
-    if (valid == 4) return ld4(q);
-    return make_float4(q[0], valid > 1 ? q[1] : 0.f, valid > 2 ? q[2] : 0.f, 0.f);
+    extern __shared__ float norm_acc[];     // [K][blockDim.x]
+    const int tid = threadIdx.x, bd = blockDim.x;
+    const int64_t n_col = (p.P + 3) >> 2;
+    const int64_t j = int64_t(blockIdx.x) * bd + tid;
+    if (j < n_col) {
+        const int64_t i0 = j << 2;
+        const int valid = i0 + 4 <= p.P ? 4 : int(p.P - i0);
+        float4 lam = make_float4(0.f, 0.f, 0.f, 0.f), ths = lam;
+        if (!EXT_GRAD) {
+            lam = ld4_guarded(p.lambda + i0, valid);
+            ths = ld4_guarded(p.theta_star + i0, valid);
+        }
+        const float *src = EXT_GRAD ? p.grads : p.theta;
+        auto one_row = [&](int k, float4 v) {
+            if (EXT_GRAD) norm_acc[k * bd + tid] = fmaf(v.x, v.x, v.y * v.y) + fmaf(v.z, v.z, v.w * v.w);   // zeros beyond P
+            else norm_acc[k * bd + tid] = column_sq(p, j, p.step, k, v, lam, ths, valid);
+        };
+        int k = 0;
+        for (; k + 4 <= p.K; k += 4) {      // four rows' loads in flight before the arithmetic of the first
+            float4 v[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) v[r] = ld4_guarded(src + int64_t(k + r) * p.stride + i0, valid);
+#pragma unroll
+            for (int r = 0; r < 4; ++r) one_row(k + r, v[r]);
+        }
+        for (; k < p.K; ++k) one_row(k, ld4_guarded(src + int64_t(k) * p.stride + i0, valid));
+    } else {
+        for (int k = 0; k < p.K; ++k) norm_acc[k * bd + tid] = 0.f;
+    }
+    __syncthreads();
+    reduce_rows_to_partials(norm_acc, p.K, partial);
 }
 
-// Pass 1 of global-norm clipping (App. C.2): partial sums of g^2, per worker (PARALLEL = false: one sum per row k of
-// the gradient that worker's step will use) or of the averaged gradient (PARALLEL = true: Algorithm 1).  Generated
-// gradients are recomputed here with the very expressions of the step kernel -- the noise is a pure function of
-// (seed, worker, step, coordinate) -- so nothing has to be stored: the pass reads theta once (4 B per update).
-// The grid is fixed (kNormGrid blocks at most) so that the partials fit a small workspace; a thread strides over
-// columns and keeps its running sum for worker k in shared memory at acc[k * blockDim.x + threadIdx.x].
-// partial is [gridDim.x, rows] with rows = PARALLEL ? 1 : K.  Summation order is fixed: results are deterministic.
-template <bool EXT_GRAD, bool PARALLEL>
-__global__ void grad_sqnorm_kernel(const __grid_constant__ StepParams p, float *partial)
+// The same pass for Algorithm 1: the squared norm of the AVERAGED gradient, all K gradients taken at the single model
+// in row 0.  The grid is fixed (kNormGrid blocks at most); a thread strides over columns and keeps a running sum.
+// partial is [gridDim.x].  Summation order is fixed: results are deterministic.
+template <bool EXT_GRAD>
+__global__ void parallel_sqnorm_kernel(const __grid_constant__ StepParams p, float *partial)
 {
     extern __shared__ float acc[];
-    const int rows = PARALLEL ? 1 : p.K;
-    for (int r = 0; r < rows; ++r) acc[r * blockDim.x + threadIdx.x] = 0.f;
+    acc[threadIdx.x] = 0.f;
     const int64_t n_col = (p.P + 3) >> 2;
     const int64_t grid_stride = int64_t(gridDim.x) * blockDim.x;
     const float Kf = float(p.K);
     for (int64_t j = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; j < n_col; j += grid_stride) {
         const int64_t i0 = j << 2;
         const int valid = i0 + 4 <= p.P ? 4 : int(p.P - i0);
-        float4 lam = make_float4(0.f, 0.f, 0.f, 0.f), ths = lam, sum = lam;
+        float4 lam = make_float4(0.f, 0.f, 0.f, 0.f), ths = lam, sum = lam, th = lam;
         if (!EXT_GRAD) {
             lam = ld4_guarded(p.lambda + i0, valid);     // zero lambda and zero noise weight make the lanes beyond P vanish
             ths = ld4_guarded(p.theta_star + i0, valid);
+            th = ld4_guarded(p.theta + i0, valid);
         }
         for (int k = 0; k < p.K; ++k) {
             float4 g;
             if (EXT_GRAD) {
                 g = ld4_guarded(p.grads + int64_t(k) * p.stride + i0, valid);
             } else {
-                // Algorithm 1 evaluates every worker's gradient at the single model in row 0
-                const float4 th = ld4_guarded(p.theta + int64_t(PARALLEL ? 0 : k) * p.stride + i0, valid);
                 const float4 z = noise4_packed(j, p.step, p.worker0 + uint32_t(k), p.round_key);
                 g = gradient4(p.sigma, z, lam, th, ths);
                 if (valid < 4) {                   // ragged last column: the lanes beyond P do not count
@@ -592,37 +677,33 @@ __global__ void grad_sqnorm_kernel(const __grid_constant__ StepParams p, float *
                     g.w = 0.f;
                 }
             }
-            if (PARALLEL) sum = add4(sum, g);
-            else acc[k * blockDim.x + threadIdx.x] += (g.x * g.x + g.y * g.y) + (g.z * g.z + g.w * g.w);
+            sum = add4(sum, g);
         }
-        if (PARALLEL) {
-            sum = div4(sum, Kf);
-            acc[threadIdx.x] += (sum.x * sum.x + sum.y * sum.y) + (sum.z * sum.z + sum.w * sum.w);
-        }
+        sum = div4(sum, Kf);
+        acc[threadIdx.x] += (sum.x * sum.x + sum.y * sum.y) + (sum.z * sum.z + sum.w * sum.w);
     }
     __syncthreads();
-    // block reduction per worker: warp w folds rows w, w + n_warps, ...
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    for (int r = warp; r < rows; r += n_warps) {
-        float v = 0.f;
-        for (int t = lane; t < int(blockDim.x); t += 32) v += acc[r * blockDim.x + t];
-        for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0) partial[int64_t(blockIdx.x) * rows + r] = v;
-    }
+    reduce_rows_to_partials(acc, 1, partial);
 }
 
-// Pass 2: coef[r] = min(1, max_norm / (sqrt(sum of partials) + 1e-6)), accumulated in binary64 in a fixed order.
-__global__ void clip_coef_kernel(const float *partial, int n_blocks, int rows, double max_norm, float *coef)
+// Pass 2: coef[r] = min(1, max_norm / (sqrt(sum of partials) + 1e-6)).  One block per row; every thread adds its
+// stride of the row's partials in binary64, then the block folds the 256 sums in a fixed tree: deterministic.
+__global__ void __launch_bounds__(256) clip_coef_kernel(const float *partial, int64_t n_blocks, int rows, double max_norm,
+                                                         float *coef)
 {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
-    for (int r = warp; r < rows; r += n_warps) {
-        double s = 0.0;
-        for (int b = lane; b < n_blocks; b += 32) s += double(partial[int64_t(b) * rows + r]);
-        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if (lane == 0) {
-            const double c = max_norm / (sqrt(s) + 1e-6);
-            coef[r] = float(c < 1.0 ? c : 1.0);
-        }
+    __shared__ double part[256];
+    const int r = blockIdx.x;
+    double s = 0.0;
+    for (int64_t b = threadIdx.x; b < n_blocks; b += 256) s += double(partial[b * rows + r]);
+    part[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o; o >>= 1) {
+        if (int(threadIdx.x) < o) part[threadIdx.x] += part[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const double c = max_norm / (sqrt(part[0]) + 1e-6);
+        coef[r] = float(c < 1.0 ? c : 1.0);
     }
 }
 
@@ -861,12 +942,12 @@ unsigned grid_for(int64_t P, int threads)
 
 // Picks one instance of the step kernel and its launch geometry; raises the instance's dynamic shared-memory limit
 // (the ring exceeds the 48 KB default).  Returns a cudaError_t as int.
-template <int OPT, bool EXT, int STAGES, int FUSE, bool EXTRAS>
+template <int OPT, bool EXT, int STAGES, int FUSE, bool EXTRAS, bool NEXTNORM>
 int resolve_step_instance(const StepParams &p, int threads, StepLaunch *out)
 {
-    const size_t smem = size_t(STAGES) * StepOperands<OPT, EXT>::kCount * threads * sizeof(float4);
+    const size_t smem = step_shared_bytes(OPT, EXT, STAGES, threads, NEXTNORM ? p.K : 0);
     if (smem > 227 * 1024) return int(cudaErrorInvalidValue);
-    auto kernel = local_step_kernel<OPT, EXT, STAGES, FUSE, EXTRAS>;
+    auto kernel = local_step_kernel<OPT, EXT, STAGES, FUSE, EXTRAS, NEXTNORM>;
     if (smem > 48 * 1024) {
         if (cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem)))
             return int(e);
@@ -878,22 +959,26 @@ int resolve_step_instance(const StepParams &p, int threads, StepLaunch *out)
     return 0;
 }
 
-template <int OPT, bool EXT, int FUSE, bool EXTRAS>
+template <int OPT, bool EXT, int FUSE, bool EXTRAS, bool NEXTNORM>
 int resolve_step_stages(const StepParams &p, const LaunchShape &s, StepLaunch *out)
 {
     switch (s.step_rows ? s.step_rows : 8) {
-    case 1: return resolve_step_instance<OPT, EXT, 1, FUSE, EXTRAS>(p, s.step_threads, out);
-    case 2: return resolve_step_instance<OPT, EXT, 2, FUSE, EXTRAS>(p, s.step_threads, out);
-    case 4: return resolve_step_instance<OPT, EXT, 4, FUSE, EXTRAS>(p, s.step_threads, out);
-    default: return resolve_step_instance<OPT, EXT, 8, FUSE, EXTRAS>(p, s.step_threads, out);
+    case 1: return resolve_step_instance<OPT, EXT, 1, FUSE, EXTRAS, NEXTNORM>(p, s.step_threads, out);
+    case 2: return resolve_step_instance<OPT, EXT, 2, FUSE, EXTRAS, NEXTNORM>(p, s.step_threads, out);
+    case 4: return resolve_step_instance<OPT, EXT, 4, FUSE, EXTRAS, NEXTNORM>(p, s.step_threads, out);
+    default: return resolve_step_instance<OPT, EXT, 8, FUSE, EXTRAS, NEXTNORM>(p, s.step_threads, out);
     }
 }
 
 template <int OPT, bool EXT, int FUSE>
 int resolve_step_extras(const StepParams &p, const LaunchShape &s, StepLaunch *out)
 {
-    if (p.n_tensors > 0 || p.clip_coef) return resolve_step_stages<OPT, EXT, FUSE, true>(p, s, out);
-    return resolve_step_stages<OPT, EXT, FUSE, false>(p, s, out);
+    if (p.norm_partial) {       // only the plain step with generated gradients computes the next norms on the side
+        if (EXT || FUSE != FUSE_NONE) return int(cudaErrorInvalidValue);
+        return resolve_step_stages<OPT, false, FUSE_NONE, true, true>(p, s, out);
+    }
+    if (p.n_tensors > 0 || p.clip_coef) return resolve_step_stages<OPT, EXT, FUSE, true, false>(p, s, out);
+    return resolve_step_stages<OPT, EXT, FUSE, false, false>(p, s, out);
 }
 
 template <int FUSE>
@@ -917,6 +1002,13 @@ int launch_resolved(const StepParams &p, int opt, const LaunchShape &shape, int 
 }
 
 }  // namespace
+
+// Dynamic shared memory of a step launch: the ring, plus K x threads floats when the next step's norms ride along.
+size_t step_shared_bytes(int opt, bool ext_grad, int stages, int threads, int next_norm_rows)
+{
+    const int operands = 1 + (opt == QSR_OPT_ADAMW ? 2 : 1) + (ext_grad ? 1 : 0);
+    return size_t(stages) * operands * threads * sizeof(float4) + size_t(next_norm_rows) * threads * sizeof(float);
+}
 
 int resolve_step(const StepParams &p, int opt, const LaunchShape &shape, int fuse, StepLaunch *out)
 {
@@ -964,26 +1056,40 @@ int clip_grid(int64_t P)
     return int(want < kNormGrid ? (want < 1 ? 1 : want) : kNormGrid);
 }
 
-// Enqueues the two clipping passes; afterwards ws[clip_grid*rows .. +rows) holds the factors.
-int launch_clip_coef(const StepParams &p, bool parallel, double max_norm, float *ws, const LaunchShape &shape, void *stream)
+// Blocks of the per-worker norm pass = blocks of a step launch with this block size: one thread per column.
+int64_t clip_norm_blocks(int64_t P, int threads) { return int64_t(grid_for(P, threads)); }
+
+// Enqueues the norm pass of Local OPT: ws[0 .. blocks * K) receives the partial sums.
+int launch_clip_norms(const StepParams &p, float *ws, const LaunchShape &shape, void *stream)
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int threads = kNormThreads;
-    const int rows = parallel ? 1 : p.K;
-    const int grid = clip_grid(p.P);
-    const size_t smem = size_t(rows) * threads * sizeof(float);
-    if (smem > 48 * 1024) return int(cudaErrorInvalidValue);
-    const bool ext = p.grads != nullptr;
-    if (parallel) {
-        if (ext) grad_sqnorm_kernel<true, true><<<grid, threads, smem, st>>>(p, ws);
-        else grad_sqnorm_kernel<false, true><<<grid, threads, smem, st>>>(p, ws);
-    } else {
-        if (ext) grad_sqnorm_kernel<true, false><<<grid, threads, smem, st>>>(p, ws);
-        else grad_sqnorm_kernel<false, false><<<grid, threads, smem, st>>>(p, ws);
-    }
-    if (cudaError_t e = cudaGetLastError()) return int(e);
-    clip_coef_kernel<<<1, 256, 0, st>>>(ws, grid, rows, max_norm, ws + int64_t(grid) * rows);
+    const int threads = shape.step_threads;
+    const size_t smem = size_t(p.K) * threads * sizeof(float);
+    if (smem > 227 * 1024) return int(cudaErrorInvalidValue);
+    auto kernel = p.grads ? column_sqnorm_kernel<true> : column_sqnorm_kernel<false>;
+    if (smem > 48 * 1024)
+        if (cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))) return int(e);
+    kernel<<<grid_for(p.P, threads), threads, smem, st>>>(p, ws);
     return int(cudaGetLastError());
+}
+
+// Enqueues the factor pass over `blocks` partials per row: ws[blocks * rows .. +rows) receives the factors.
+int launch_clip_factors(float *ws, int64_t blocks, int rows, double max_norm, void *stream)
+{
+    clip_coef_kernel<<<unsigned(rows), 256, 0, static_cast<cudaStream_t>(stream)>>>(ws, blocks, rows, max_norm, ws + blocks * rows);
+    return int(cudaGetLastError());
+}
+
+// Algorithm 1: both clipping passes; afterwards ws[clip_grid(P)] holds the factor.
+int launch_clip_coef_parallel(const StepParams &p, double max_norm, float *ws, void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int grid = clip_grid(p.P);
+    const size_t smem = size_t(kNormThreads) * sizeof(float);
+    if (p.grads) parallel_sqnorm_kernel<true><<<grid, kNormThreads, smem, st>>>(p, ws);
+    else parallel_sqnorm_kernel<false><<<grid, kNormThreads, smem, st>>>(p, ws);
+    if (cudaError_t e = cudaGetLastError()) return int(e);
+    return launch_clip_factors(ws, grid, 1, max_norm, stream);
 }
 
 // The state slabs a synchronization resets: a launch of its own after the averaging (see rows_kernel).

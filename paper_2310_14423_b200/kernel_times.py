@@ -102,6 +102,18 @@ def main(argv=None):
     ws = torch.zeros(ctx.qsr_clip_workspace_floats(), device=dev)
     ctx.qsr_set_grad_clip(1.0, ws)
     add("clipped local step (norm pass + factors + step: three launches)", timed(step), (n_slabs * 8 + 4 + 16 / w.K) * KP)
+    # inside qsr_run a step leaves its successor's norm partials behind: time a whole round and divide by its steps
+    t_round = [0]
+
+    def clipped_round():
+        st_, H_ = ctx.qsr_run(0, 1)
+        t_round[0] = int(H_[0])
+
+    saved, args.launches = args.launches, max(1, args.launches // 10)
+    ms_round = timed(clipped_round)
+    args.launches = saved
+    add(f"clipped local step inside qsr_run (round of {t_round[0]} steps; factors + step, norm pass once per round)",
+        ms_round / t_round[0], (n_slabs * 8 + 8 / w.K) * KP)
     add("clipped Algorithm-1 step (row 0; three launches)", timed(parallel), evals=2 * KP)
     ctx.qsr_set_grad_clip(0.0)
     add("Algorithm-1 step (row 0, K gradients per coordinate)", timed(parallel), evals=KP)

@@ -34,7 +34,9 @@ def test_clipped_local_runs(opt, K, P):
     ctx, ws = _clip_context(w, S, lam_d, ths_d)
     st, H = ctx.qsr_run()
     torch.cuda.synchronize()
-    assert ctx.qsr_launch_count() == 3 * w.T              # norm pass, factor pass, step
+    # per step the factor pass and the step; the norm pass only at a round's first step (later steps find the partial
+    # sums their predecessor left behind)
+    assert ctx.qsr_launch_count() == 2 * w.T + len(st)
     orc = G.oracle_on(w, lam, ths)
     ost, oH = orc.run()
     assert np.array_equal(st, ost) and np.array_equal(H, oH)
@@ -109,3 +111,55 @@ def test_clip_switch_and_argument_errors():
     assert ctx.qsr_launch_count() == 4
     torch.cuda.synchronize()
     ctx.close()
+
+
+@pytest.mark.parametrize("opt", [W.OPT_SGDM, W.OPT_ADAMW])
+@pytest.mark.parametrize("K,P,mode", [(1, 3, W.STATE_KEEP), (3, 1001, W.STATE_KEEP), (16, 40002, W.STATE_KEEP),
+                                      (5, 70003, W.STATE_RESET), (7, 4100, W.STATE_AVERAGE)])
+def test_norms_left_by_the_previous_step_equal_the_norm_pass_bitwise(opt, K, P, mode):
+    """Inside qsr_run a plain step also computes its successor's gradient-norm partials; driving the same steps one
+    call at a time runs the stand-alone norm pass before every step.  The two must agree in every bit of every slab:
+    same per-column values, same block geometry, same order of summation."""
+    clip = {3: 0.02, 1001: 3.0, 40002: 20.0, 70003: 25.0, 4100: 6.0}[P]
+    w = W.tiny_workload(opt, K=K, P=P, T=60, clip_norm=clip, state_sync=mode)
+    lam, ths, lam_d, ths_d = G.device_inputs(w)
+    A, Bs = G.Slabs(w), G.Slabs(w)
+    ca, wa = _clip_context(w, A, lam_d, ths_d)
+    cb, wb = _clip_context(w, Bs, lam_d, ths_d)
+    st, H = ca.qsr_run()
+    t = 0
+    while t < w.T:
+        h = cb.qsr_round_length(t)
+        for u in range(t, t + h - 1):
+            cb.qsr_local_step(u)
+        cb.qsr_local_step_sync(t + h - 1, t + h)
+        t += h
+    torch.cuda.synchronize()
+    assert cb.qsr_launch_count() > ca.qsr_launch_count()
+    assert torch.equal(A.theta, Bs.theta) and torch.equal(A.s1, Bs.s1)
+    assert A.s2 is None or torch.equal(A.s2, Bs.s2)
+    assert A.guards_intact() and Bs.guards_intact() and bool((wa[-8:] == 7.0).all())
+    # and clipping was active on some steps but not on all: the factors in the workspace are not all 1
+    ca.close()
+    cb.close()
+
+
+def test_norms_fall_back_to_the_norm_pass_when_the_block_has_no_room():
+    """K x threads sums must fit next to the step's ring in shared memory; with 512-thread blocks and K = 96 (the most
+    clipping takes) AdamW's 96 KiB ring (four rows in flight) leaves no room for 192 KiB more, so every step runs the
+    stand-alone norm pass -- with the same result up to the order of the norms' partial sums."""
+    w = W.tiny_workload(W.OPT_ADAMW, K=96, P=3001, T=24, clip_norm=6.0)
+    lam, ths, lam_d, ths_d = G.device_inputs(w)
+    for threads in (256, 512):
+        S = G.Slabs(w)
+        ctx, ws = _clip_context(w, S, lam_d, ths_d)
+        ctx.qsr_set_launch_shape(threads, 4, 0)
+        st, H = ctx.qsr_run()
+        torch.cuda.synchronize()
+        expect = 2 * w.T + len(st) if threads == 256 else 3 * w.T
+        assert ctx.qsr_launch_count() == expect
+        orc = G.oracle_on(w, lam, ths)
+        orc.run()
+        G.assert_parity(S.theta[0, :w.P].cpu().numpy(), w, lam, ths, orc.theta[0])
+        assert S.guards_intact() and bool((ws[-8:] == 7.0).all())
+        ctx.close()
