@@ -148,7 +148,8 @@ class ClockSampler:
         return out
 
     def stop(self, t0: float, t1: float):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "period_ms": self.PERIOD_MS}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "source": "nvidia-smi",
+               "period_ms": self.PERIOD_MS}
         if self.proc is None:
             return out
         time.sleep(2e-3 * self.PERIOD_MS)          # let the sample that covers the end of the region be written
@@ -172,6 +173,61 @@ class ClockSampler:
             reasons = set().union(*[r[3] for r in rows])
             out.update(sm_mhz=float(np.median([r[0] for r in rows])), sm_max_mhz=float(max(r[1] for r in rows)),
                        reasons=sorted(reasons), samples=len(rows), power_w_median=float(np.median([r[2] for r in rows])))
+        return out
+
+
+class NvmlSampler:
+    """The same record from NVML inside this process: a thread reads the SM clock, the power draw and the clock event
+    reasons every few milliseconds (read-only queries).  The timed loop only enqueues kernels and then waits in
+    cudaDeviceSynchronize with the interpreter lock released, so the thread runs freely and even the 0.1 s of a
+    20-step window gets a dozen readings taken under its own load.  `stop(t0, t1)` keeps those stamped inside the
+    region.  Raises if NVML cannot be used; the caller then falls back to the nvidia-smi sampler."""
+    PERIOD_S = 0.005
+
+    def __init__(self, gpu_uuid: str):
+        import threading
+        import pynvml
+        self.nv = pynvml
+        pynvml.nvmlInit()
+        self.h = pynvml.nvmlDeviceGetHandleByUUID(gpu_uuid.encode() if hasattr(gpu_uuid, "encode") else gpu_uuid)
+        self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        self.rows = []
+        self.halt = threading.Event()
+        self._read()                                  # fail here, not in the thread, if a query is unsupported
+        self.thread = threading.Thread(target=self._loop, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        nv = self.nv
+        mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+        names = {"hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown,
+                 "hw_thermal_slowdown": nv.nvmlClocksEventReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": nv.nvmlClocksEventReasonSwThermalSlowdown,
+                 "sw_power_cap": nv.nvmlClocksEventReasonSwPowerCap}
+        return (time.time(), float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)),
+                float(nv.nvmlDeviceGetPowerUsage(self.h)) / 1e3, {n for n, bit in names.items() if mask & bit})
+
+    def _loop(self):
+        while not self.halt.is_set():
+            try:
+                self.rows.append(self._read())
+            except Exception:
+                break
+            self.halt.wait(self.PERIOD_S)
+
+    def stop(self, t0: float, t1: float):
+        self.halt.set()
+        self.thread.join(timeout=2)
+        out = {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": [], "samples": 0, "source": "nvml",
+               "period_ms": 1e3 * self.PERIOD_S}
+        rows = [r for r in self.rows if t0 <= r[0] <= t1]
+        if rows:
+            out.update(sm_mhz=float(np.median([r[1] for r in rows])), reasons=sorted(set().union(*[r[3] for r in rows])),
+                       samples=len(rows), power_w_median=float(np.median([r[2] for r in rows])))
+        try:
+            self.nv.nvmlShutdown()
+        except Exception:
+            pass
         return out
 
 
@@ -289,8 +345,11 @@ class CudaBackend:
         self.torch.cuda.empty_cache()
 
     def clock_sampler(self):
-        uuid = str(self.torch.cuda.get_device_properties(self.local_rank).uuid)
-        return ClockSampler("GPU-" + uuid.replace("GPU-", ""))
+        uuid = "GPU-" + str(self.torch.cuda.get_device_properties(self.local_rank).uuid).replace("GPU-", "")
+        try:
+            return NvmlSampler(uuid)
+        except Exception:
+            return ClockSampler(uuid)
 
 
 def rank_layout(base, world: int, rank: int):
