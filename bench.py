@@ -221,6 +221,12 @@ class NvmlSampler:
         out = {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": [], "samples": 0, "source": "nvml",
                "period_ms": 1e3 * self.PERIOD_S}
         rows = [r for r in self.rows if t0 <= r[0] <= t1]
+        if not rows and self.rows:
+            # a region shorter than the period can fall between two readings: take the nearest one
+            nearest = min(self.rows, key=lambda r: min(abs(r[0] - t0), abs(r[0] - t1)))
+            if min(abs(nearest[0] - t0), abs(nearest[0] - t1)) <= 4 * self.PERIOD_S:
+                rows = [nearest]
+                out["note"] = "the timed region fell between two readings; this is the nearest one"
         if rows:
             out.update(sm_mhz=float(np.median([r[1] for r in rows])), reasons=sorted(set().union(*[r[3] for r in rows])),
                        samples=len(rows), power_w_median=float(np.median([r[2] for r in rows])))
