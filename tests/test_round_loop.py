@@ -104,3 +104,46 @@ def test_clock_samples_are_filtered_by_their_time_stamps():
     assert bench.ClockSampler.parse(lines, t0 + 0.2, t0 + 0.25) == []
     near = bench.ClockSampler.parse(lines, t0 + 0.2, t0 + 0.25, slack_s=0.06)
     assert [r[0] for r in near] == [1965.0]
+
+
+def test_nvml_sampler_keeps_the_readings_inside_the_region(monkeypatch):
+    """The in-process clock sampler against a stand-in for the NVML binding: readings every few milliseconds, only
+    those stamped inside the timed region are kept, reasons come from the bit mask, and a region shorter than the
+    period takes the nearest reading."""
+    import time
+    import types
+    import bench
+    calls = {"n": 0}
+    fake = types.ModuleType("pynvml")
+    fake.NVML_CLOCK_SM = 1
+    fake.nvmlClocksEventReasonHwSlowdown, fake.nvmlClocksEventReasonHwThermalSlowdown = 0x8, 0x40
+    fake.nvmlClocksEventReasonSwThermalSlowdown, fake.nvmlClocksEventReasonSwPowerCap = 0x20, 0x4
+    fake.nvmlInit = lambda: None
+    fake.nvmlShutdown = lambda: None
+    fake.nvmlDeviceGetHandleByUUID = lambda uuid: ("handle", uuid)
+    fake.nvmlDeviceGetMaxClockInfo = lambda h, which: 1965
+
+    def clock(h, which):
+        calls["n"] += 1
+        return 1500 if calls["n"] > 3 else 1965
+
+    fake.nvmlDeviceGetClockInfo = clock
+    fake.nvmlDeviceGetPowerUsage = lambda h: 990000
+    fake.nvmlDeviceGetCurrentClocksEventReasons = lambda h: 0x4 if calls["n"] > 3 else 0x1
+    monkeypatch.setitem(sys.modules, "pynvml", fake)
+    s = bench.NvmlSampler("GPU-00000000-0000-0000-0000-000000000000")
+    time.sleep(0.03)
+    t0 = time.time()
+    time.sleep(0.08)
+    t1 = time.time()
+    time.sleep(0.02)
+    out = s.stop(t0, t1)
+    assert out["source"] == "nvml" and out["sm_max_mhz"] == 1965.0
+    assert 5 <= out["samples"] <= 20 and out["sm_mhz"] == 1500.0 and out["reasons"] == ["sw_power_cap"]
+    assert out["power_w_median"] == 990.0
+    # a region between two readings
+    s = bench.NvmlSampler("GPU-00000000-0000-0000-0000-000000000000")
+    time.sleep(0.03)
+    t0 = time.time()
+    out = s.stop(t0, t0 + 1e-4)
+    assert out["samples"] == 1 and "note" in out
