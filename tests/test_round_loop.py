@@ -139,7 +139,7 @@ def test_nvml_sampler_keeps_the_readings_inside_the_region(monkeypatch):
     time.sleep(0.02)
     out = s.stop(t0, t1)
     assert out["source"] == "nvml" and out["sm_max_mhz"] == 1965.0
-    assert 5 <= out["samples"] <= 20 and out["sm_mhz"] == 1500.0 and out["reasons"] == ["sw_power_cap"]
+    assert 3 <= out["samples"] <= 20 and out["sm_mhz"] == 1500.0 and out["reasons"] == ["sw_power_cap"]
     assert out["power_w_median"] == 990.0
     # a region between two readings
     s = bench.NvmlSampler("GPU-00000000-0000-0000-0000-000000000000")
