@@ -255,3 +255,18 @@ def test_train_host_fails_before_touching_a_device_and_zeroes_its_outputs():
     if not torch.cuda.is_available():
         # a valid call on a machine without a device: the context cannot be created, nothing was enqueued
         assert call(cfg) == (B.QSR_ECUDA, 0, 0)
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/qsr.h is a C header: plain pointers and sizes, no C++ in the signatures.  gcc -std=c99 -pedantic must take it."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler here")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "use_header.c"
+    src.write_text('#include "include/qsr.h"\nint main(void) { qsr_config c; (void)c; return QSR_OK; }\n')
+    r = subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-I", root, str(src)],
+                       capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
